@@ -1,0 +1,153 @@
+/*
+ * sjd.h -- C ABI of the SJD / SJD++ verify-and-redraft step for NVIDIA B200 (sm_100a).
+ *
+ * One call of sjd_step() is one speculative Jacobi iteration's sampling and verification work for B
+ * sequences with a window of W draft image tokens each, over a V-token vocabulary:
+ *
+ *   sampling head   merged = uncond + s (cond - uncond), y = merged / T, top-K filter, softmax over the
+ *                   survivors (paper Section 3.1; K and the guidance weight s in Section 5.1)
+ *   verification    accept draft x_i iff r < min(1, p_i(x_i) / q_i(x_i)), r ~ U[0,1)  (Eq. acc-sjdpp);
+ *                   everything from the first failed test on is rejected (Section 4.1, Step 4)
+ *   residual        the first rejected position is redrawn from max(0, p - q) / sum max(0, p - q)
+ *                   (Eq. rej-sjd)
+ *   redraft         later positions keep their draft when C_i = p_i(x_i)/q_i(x_i) > tau (Eq. reuse, the
+ *                   SJD++ rule) and are otherwise redrawn from p_i; with SJD_FLAG_REUSE off every later
+ *                   position is redrawn (plain SJD, Eq. refine-sjd)
+ *
+ * p_i is this call's distribution at window row i, q_i the distribution the draft was drawn from in the
+ * previous iteration.  Distributions cross the ABI in sparse form: after top-K a row has at most
+ * kcap = min(top_k, V) non-zero entries, stored as ascending token ids plus probabilities.
+ *
+ * All arithmetic runs in the library's CUDA kernels.  The library allocates nothing, frees nothing and
+ * never synchronises in sjd_step(): the caller owns every buffer, including the scratch workspace, and
+ * the call returns as soon as the kernels are enqueued on params->stream.
+ *
+ * Random numbers: Philox4x32-10, key = (seed low word, seed high word), counter = (absolute position,
+ * sequence index, Jacobi iteration, purpose); one block per decision, no state.  A uniform for the accept
+ * test is (x0 >> 8) * 2^-24.  Sampling uses a fixed-point inverse CDF: weight w_k -> floor(w_k * 2^40),
+ * T = sum, t = floor((x0 | x1 << 32) * T / 2^64), result = first entry (ascending token id) whose running
+ * sum exceeds t.
+ *
+ * Unless stated otherwise every pointer below is a DEVICE pointer valid on the device that is current
+ * when the call is made.  No entry point throws; errors are reported by the return value.
+ */
+#ifndef SJD_H_
+#define SJD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SJD_VERSION 1
+#define SJD_W_MAX 512 /* largest window of the paper's window-size ablation */
+
+/* logits_dtype */
+#define SJD_F32 0
+#define SJD_BF16 1
+
+/* flags */
+#define SJD_FLAG_REUSE 1     /* Eq. reuse (SJD++); clear = Eq. refine-sjd (SJD)                              */
+#define SJD_FLAG_DRAFT_ALL 2 /* no verification: draw every valid row from its own p (initial drafts; Section
+                                4.2 strategies that sample from a predicted distribution).  accept_len = 0. */
+
+/* cnt value of a row of sjd_probs that stands for the uniform distribution over V (1/V each); used for
+ * window slots that were initialised at random and have no previous-iteration distribution. */
+#define SJD_Q_UNIFORM (-1)
+
+/* out_flags values */
+#define SJD_OUT_INVALID 0   /* row >= win_len                         */
+#define SJD_OUT_ACCEPTED 1  /* draft kept, part of the accepted prefix */
+#define SJD_OUT_RESIDUAL 2  /* first rejected row, residual sample     */
+#define SJD_OUT_REUSED 3    /* draft kept by the confidence rule       */
+#define SJD_OUT_RESAMPLED 4 /* redrawn from p_i                        */
+
+/* status bits (per sequence, OR-ed) */
+#define SJD_STATUS_QTOK_NONPOSITIVE 1 /* q_i(x_i) <= 0 at a valid row: treated as an infinite ratio      */
+#define SJD_STATUS_EMPTY_RESIDUAL 2   /* fixed-point residual total was 0: drawn from p instead          */
+#define SJD_STATUS_DEGENERATE_ROW 4   /* a row had no finite logit: its probabilities are all 0          */
+
+/* return codes */
+#define SJD_OK 0
+#define SJD_ERR_NULL (-1)      /* a required pointer is NULL                                              */
+#define SJD_ERR_SHAPE (-2)     /* B < 0, W outside 1..SJD_W_MAX, V < 8 or not a multiple of 8, top_k < 1  */
+#define SJD_ERR_ALIGN (-3)     /* logits base or strides not 16-byte aligned                              */
+#define SJD_ERR_DTYPE (-4)     /* unknown logits_dtype                                                    */
+#define SJD_ERR_WORKSPACE (-5) /* workspace NULL, misaligned or smaller than sjd_workspace_bytes()        */
+#define SJD_ERR_STRUCT (-6)    /* params->struct_size does not match this header                          */
+#define SJD_ERR_CUDA (-7)      /* a CUDA runtime call failed (see sjd_last_cuda_error)                    */
+#define SJD_ERR_CAPACITY (-8)  /* a fixed-capacity entry point was given a problem beyond its limit       */
+
+/* A set of per-position distributions plus the probability of one designated token per position.
+ * Row r = b*W + i.  Rows at or beyond a sequence's win_len have cnt = 0. */
+typedef struct {
+  float* tok_prob; /* [B,W]       probability of the token in the matching token array (drafts / out_tokens) */
+  int32_t* ids;    /* [B,W,kcap]  support of the row, ascending token id                                     */
+  float* vals;     /* [B,W,kcap]  probabilities on that support                                              */
+  int32_t* cnt;    /* [B,W]       entries used (kcap for a valid row), or SJD_Q_UNIFORM on input             */
+} sjd_probs;
+
+/* HOST struct, read during the call; device pointers inside it are read by the kernels. */
+typedef struct {
+  int32_t struct_size;        /* sizeof(sjd_params)                                                        */
+  int32_t B, W, V;            /* sequences, window rows, vocabulary                                        */
+  int32_t logits_dtype;       /* SJD_F32 or SJD_BF16                                                       */
+  int64_t stride_b, stride_w; /* element strides of BOTH logits tensors; the vocabulary axis is contiguous;
+                                 stride * element size must be a multiple of 16 bytes                      */
+  float cfg_scale;            /* s; unused when logits_uncond is NULL                                      */
+  float inv_temperature;      /* 1/T, rounded to float by the caller; 1.0f is an exact no-op               */
+  int32_t top_k;              /* K >= 1; kcap = min(K, V)                                                  */
+  float reuse_tau;            /* tau of Eq. reuse (the paper uses 0.5)                                     */
+  int32_t flags;              /* SJD_FLAG_*                                                                */
+  int32_t iteration0;         /* Jacobi iteration index used when `iteration` is NULL                      */
+  const int32_t* win_len;     /* [B] device, valid rows per sequence (ragged windows); NULL = W            */
+  const int32_t* pos_base;    /* [B] device, absolute image-token index of window row 0; NULL = 0          */
+  const int32_t* iteration;   /* [B] device, per-sequence iteration index; NULL = iteration0               */
+  int32_t* out_flags;         /* [B,W] device, optional SJD_OUT_* per position                             */
+  int32_t* status;            /* [B] device, optional SJD_STATUS_* bits per sequence (overwritten)         */
+  void* workspace;            /* device scratch, 256-byte aligned, owned by the caller                     */
+  size_t workspace_bytes;     /* >= sjd_workspace_bytes(params)                                            */
+  void* stream;               /* cudaStream_t the work is enqueued on (NULL = legacy default stream)       */
+} sjd_params;
+
+/* Library version (SJD_VERSION of the build). */
+int sjd_version(void);
+
+/* Static text for a return code. */
+const char* sjd_status_string(int code);
+
+/* Text of the last CUDA runtime error seen by this thread's most recent failing call ("" if none). */
+const char* sjd_last_cuda_error(void);
+
+/* Scratch bytes sjd_step() needs for this shape (depends on B, W only).  0 on a NULL argument. */
+size_t sjd_workspace_bytes(const sjd_params* params);
+
+/*
+ * One verify-and-redraft step (Section 4.1 Steps 3-4 on top of the Section 3.1 sampling head).
+ *
+ *   logits_cond    [B,W,V] device, dtype per params; row (b,i) holds the model's logits for window row i
+ *   logits_uncond  same layout, or NULL for no guidance (merged = cond)
+ *   drafts         [B,W] device int32, draft token x_i of every row          (ignored with DRAFT_ALL)
+ *   draft_probs    HOST struct of device arrays: q_i(x_i) in tok_prob and the full previous-iteration
+ *                  rows q_i in ids/vals/cnt (needed at the first rejected row)  (ignored with DRAFT_ALL)
+ *   philox_seed    key of the counter-based generator
+ *   out_accept_len [B] device int32: a_b = number of leading rows whose test passed, 0..win_len_b
+ *   out_tokens     [B,W] device int32: row < a: the draft; row a: residual sample; a < row < win_len:
+ *                  reused draft or new sample; row >= win_len: -1
+ *   out_probs      HOST struct of device arrays: tok_prob = p_i(out_tokens); ids/vals/cnt = p_i of every
+ *                  valid row.  After the caller shifts the window it is a valid draft_probs for the next
+ *                  iteration.  Must not alias draft_probs or the logits.
+ *
+ * Asynchronous on params->stream.  Returns SJD_OK once the kernels are enqueued, or a negative SJD_ERR_*
+ * with nothing enqueued.  Conditions found on the device (status bits) never abort the kernels.
+ */
+int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* drafts,
+             const sjd_probs* draft_probs, const sjd_params* params, uint64_t philox_seed,
+             int32_t* out_accept_len, int32_t* out_tokens, sjd_probs* out_probs);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SJD_H_ */

@@ -1,0 +1,178 @@
+"""Thin ctypes binding of the C ABI in ``include/sjd.h``.
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.  PyTorch is used
+for device memory and streams.  There is no CPU fallback: if the shared library cannot be built or
+loaded, importing a symbol from it raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+SJD_F32, SJD_BF16 = 0, 1
+SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL = 1, 2
+SJD_Q_UNIFORM = -1
+SJD_OUT_INVALID, SJD_OUT_ACCEPTED, SJD_OUT_RESIDUAL, SJD_OUT_REUSED, SJD_OUT_RESAMPLED = 0, 1, 2, 3, 4
+SJD_STATUS_QTOK_NONPOSITIVE, SJD_STATUS_EMPTY_RESIDUAL, SJD_STATUS_DEGENERATE_ROW = 1, 2, 4
+SJD_W_MAX = 512
+
+
+class sjd_probs(C.Structure):
+    _fields_ = [("tok_prob", C.c_void_p), ("ids", C.c_void_p), ("vals", C.c_void_p), ("cnt", C.c_void_p)]
+
+
+class sjd_params(C.Structure):
+    _fields_ = [("struct_size", C.c_int32), ("B", C.c_int32), ("W", C.c_int32), ("V", C.c_int32),
+                ("logits_dtype", C.c_int32), ("stride_b", C.c_int64), ("stride_w", C.c_int64),
+                ("cfg_scale", C.c_float), ("inv_temperature", C.c_float), ("top_k", C.c_int32),
+                ("reuse_tau", C.c_float), ("flags", C.c_int32), ("iteration0", C.c_int32),
+                ("win_len", C.c_void_p), ("pos_base", C.c_void_p), ("iteration", C.c_void_p),
+                ("out_flags", C.c_void_p), ("status", C.c_void_p), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p)]
+
+
+class SjdError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded CUDA library; built in-tree with nvcc when missing or stale.  Raises when that fails."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = C.CDLL(path)
+        L.sjd_version.restype = C.c_int
+        L.sjd_status_string.argtypes = [C.c_int]
+        L.sjd_status_string.restype = C.c_char_p
+        L.sjd_last_cuda_error.restype = C.c_char_p
+        L.sjd_workspace_bytes.argtypes = [C.POINTER(sjd_params)]
+        L.sjd_workspace_bytes.restype = C.c_size_t
+        L.sjd_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs), C.POINTER(sjd_params),
+                               C.c_uint64, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs)]
+        L.sjd_step.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def sjd_version() -> int:
+    return int(lib().sjd_version())
+
+
+def sjd_status_string(code: int) -> str:
+    return lib().sjd_status_string(int(code)).decode()
+
+
+def _check(code: int) -> None:
+    if code != 0:
+        extra = lib().sjd_last_cuda_error().decode()
+        raise SjdError(f"sjd error {code}: {sjd_status_string(code)}" + (f" ({extra})" if extra else ""))
+
+
+@dataclass
+class DeviceProbs:
+    """Device arrays of one ``sjd_probs``: tok_prob [B,W] f32, ids [B,W,kcap] i32, vals [B,W,kcap] f32, cnt [B,W] i32."""
+    tok_prob: torch.Tensor
+    ids: torch.Tensor
+    vals: torch.Tensor
+    cnt: torch.Tensor
+
+    @staticmethod
+    def empty(B: int, W: int, kcap: int, device) -> "DeviceProbs":
+        return DeviceProbs(torch.zeros(B, W, dtype=torch.float32, device=device),
+                           torch.zeros(B, W, kcap, dtype=torch.int32, device=device),
+                           torch.zeros(B, W, kcap, dtype=torch.float32, device=device),
+                           torch.zeros(B, W, dtype=torch.int32, device=device))
+
+    @staticmethod
+    def uniform(B: int, W: int, kcap: int, V: int, device) -> "DeviceProbs":
+        p = DeviceProbs.empty(B, W, kcap, device)
+        p.cnt.fill_(SJD_Q_UNIFORM)
+        p.tok_prob.fill_(1.0 / V)
+        return p
+
+    def c_struct(self) -> sjd_probs:
+        for t, dt in ((self.tok_prob, torch.float32), (self.ids, torch.int32), (self.vals, torch.float32),
+                      (self.cnt, torch.int32)):
+            if not (t.is_cuda and t.is_contiguous() and t.dtype == dt):
+                raise SjdError("sjd_probs arrays must be contiguous CUDA tensors of the documented dtypes")
+        return sjd_probs(self.tok_prob.data_ptr(), self.ids.data_ptr(), self.vals.data_ptr(), self.cnt.data_ptr())
+
+
+def _opt_ptr(t: Optional[torch.Tensor], dtype=torch.int32) -> Optional[int]:
+    if t is None:
+        return None
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise SjdError("optional arrays must be contiguous CUDA tensors of the documented dtype")
+    return t.data_ptr()
+
+
+def make_params(logits: torch.Tensor, *, top_k: int, cfg_scale: float = 1.0, inv_temperature: float = 1.0,
+                reuse_tau: float = 0.5, flags: int = SJD_FLAG_REUSE, iteration0: int = 0,
+                win_len: Optional[torch.Tensor] = None, pos_base: Optional[torch.Tensor] = None,
+                iteration: Optional[torch.Tensor] = None, out_flags: Optional[torch.Tensor] = None,
+                status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                stream: Optional[torch.cuda.Stream] = None) -> sjd_params:
+    """Fill an ``sjd_params`` from a [B,W,V] logits tensor (fp32 or bf16, vocabulary axis contiguous)."""
+    if logits.dim() != 3 or logits.stride(2) != 1:
+        raise SjdError("logits must be [B,W,V] with a contiguous vocabulary axis")
+    if logits.dtype == torch.float32:
+        dt = SJD_F32
+    elif logits.dtype == torch.bfloat16:
+        dt = SJD_BF16
+    else:
+        raise SjdError("logits must be float32 or bfloat16")
+    B, W, V = logits.shape
+    p = sjd_params()
+    p.struct_size = C.sizeof(sjd_params)
+    p.B, p.W, p.V = B, W, V
+    p.logits_dtype = dt
+    p.stride_b, p.stride_w = logits.stride(0), logits.stride(1)
+    p.cfg_scale = cfg_scale
+    p.inv_temperature = inv_temperature
+    p.top_k = top_k
+    p.reuse_tau = reuse_tau
+    p.flags = flags
+    p.iteration0 = iteration0
+    p.win_len = _opt_ptr(win_len)
+    p.pos_base = _opt_ptr(pos_base)
+    p.iteration = _opt_ptr(iteration)
+    p.out_flags = _opt_ptr(out_flags)
+    p.status = _opt_ptr(status)
+    if workspace is not None:
+        p.workspace = workspace.data_ptr()
+        p.workspace_bytes = workspace.numel() * workspace.element_size()
+    s = stream if stream is not None else torch.cuda.current_stream(logits.device)
+    p.stream = s.cuda_stream
+    return p
+
+
+def sjd_workspace_bytes(params: sjd_params) -> int:
+    return int(lib().sjd_workspace_bytes(C.byref(params)))
+
+
+def sjd_step(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor], drafts: Optional[torch.Tensor],
+             draft_probs: Optional[DeviceProbs], params: sjd_params, philox_seed: int, out_accept_len: torch.Tensor,
+             out_tokens: torch.Tensor, out_probs: DeviceProbs) -> None:
+    """Enqueue one verify-and-redraft step on ``params.stream``.  Same arguments as the C entry point."""
+    if not logits_cond.is_cuda:
+        raise SjdError("logits must live on a CUDA device")
+    if logits_uncond is not None and (logits_uncond.shape != logits_cond.shape or
+                                      logits_uncond.stride() != logits_cond.stride() or
+                                      logits_uncond.dtype != logits_cond.dtype):
+        raise SjdError("cond and uncond logits must share shape, strides and dtype")
+    q = draft_probs.c_struct() if draft_probs is not None else None
+    o = out_probs.c_struct()
+    with torch.cuda.device(logits_cond.device):
+        code = lib().sjd_step(logits_cond.data_ptr(), None if logits_uncond is None else logits_uncond.data_ptr(),
+                              _opt_ptr(drafts), C.byref(q) if q is not None else None, C.byref(params),
+                              int(philox_seed) & 0xFFFFFFFFFFFFFFFF, _opt_ptr(out_accept_len), _opt_ptr(out_tokens),
+                              C.byref(o))
+    _check(code)

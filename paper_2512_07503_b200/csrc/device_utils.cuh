@@ -1,0 +1,264 @@
+// Device-side building blocks shared by the kernels of the step: Philox4x32-10, the order-preserving
+// key of a float, logit loads with the guidance merge, and block-wide scans / reductions that work on
+// any group of NT threads synchronised by a named barrier.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sjd {
+
+constexpr int kPurposeAccept = 0;
+constexpr int kPurposeResidual = 1;
+constexpr int kPurposeRedraft = 2;
+constexpr int kPurposeInit = 3;
+
+constexpr int kRowStatusDegenerate = 1;
+
+// ------------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): counter = (position, sequence, iteration, purpose),
+// key = (seed low, seed high).
+// ------------------------------------------------------------------------------------------------
+struct Philox4 {
+  uint32_t x0, x1, x2, x3;
+};
+
+__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                                 uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0;
+    const uint32_t n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return Philox4{c0, c1, c2, c3};
+}
+
+__device__ __forceinline__ float uniform24(uint32_t x) { return (float)(x >> 8) * (1.0f / 16777216.0f); }
+
+__device__ __forceinline__ uint64_t random64(const Philox4& p) { return (uint64_t)p.x0 | ((uint64_t)p.x1 << 32); }
+
+// ------------------------------------------------------------------------------------------------
+// Order-preserving map float -> uint32 (larger float <=> larger key); -0 is folded into +0 and NaN
+// ranks with -inf before the key is taken.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float canonical(float y) {
+  if (!(y == y)) return __int_as_float(0xff800000);  // NaN -> -inf
+  return __fadd_rn(y, 0.0f);                         // -0 -> +0
+}
+
+__device__ __forceinline__ uint32_t float_key(float y) {
+  const uint32_t b = __float_as_uint(y);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Guidance merge and temperature with one rounding per operation (the result decides the top-K set):
+// d = c - u; g = fma(s, d, u); y = g * inv_T.
+__device__ __forceinline__ float merge_logit(float c, float u, float s, float inv_T) {
+  const float d = __fsub_rn(c, u);
+  const float g = __fmaf_rn(s, d, u);
+  return __fmul_rn(g, inv_T);
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Eight consecutive logits starting at element `e` (a multiple of 8) of a row, converted to fp32.
+template <int DTYPE>
+__device__ __forceinline__ void load8(const void* __restrict__ row, int e, float (&x)[8]) {
+  if (DTYPE == 1) {
+    const uint4 w = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(row) + e));
+    x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
+    x[4] = bf16_lo(w.z); x[5] = bf16_hi(w.z); x[6] = bf16_lo(w.w); x[7] = bf16_hi(w.w);
+  } else {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(row) + e));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(row) + e) + 1);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  }
+}
+
+// y of eight consecutive vocabulary entries (canonical form).
+template <int DTYPE>
+__device__ __forceinline__ void load_y8(const void* __restrict__ cond, const void* __restrict__ uncond, int e, float s,
+                                        float inv_T, float (&y)[8]) {
+  float c[8];
+  load8<DTYPE>(cond, e, c);
+  if (uncond != nullptr) {
+    float u[8];
+    load8<DTYPE>(uncond, e, u);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) y[j] = canonical(merge_logit(c[j], u[j], s, inv_T));
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) y[j] = canonical(__fmul_rn(c[j], inv_T));
+  }
+}
+
+// exp(y - m) for y <= m with the rounding error of the fp32 subtraction compensated, so that the
+// result is within a few ulp of the exact exponential of the exact difference.
+__device__ __forceinline__ float exp_diff(float y, float m) {
+  if (y == __int_as_float(0xff800000)) return 0.0f;
+  const float t = __fsub_rn(y, m);
+  const float bb = __fsub_rn(t, y);                                       // ~ -m
+  const float err = __fadd_rn(__fsub_rn(y, __fsub_rn(t, bb)), __fsub_rn(-m, bb));  // (y - m) - t, exact
+  const float e = expf(t);
+  return __fmaf_rn(e, err, e);
+}
+
+// Fixed-point weight of the inverse-CDF sampler: floor(w * 2^40) for w >= 0, 0 otherwise.
+__device__ __forceinline__ uint64_t fixed_weight(float w) {
+  return w > 0.0f ? __float2ull_rz(__fmul_rn(w, 1099511627776.0f)) : 0ull;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Group-wide primitives.  A "group" is NT threads (a multiple of 32) of one CTA whose ranks 0..NT-1
+// are passed in as `tid`; they synchronise on named barrier BAR so that other warps of the CTA
+// (copy producers) are not involved.  `scratch` points to at least 2*(NT/32)+2 uint64 slots.
+// ------------------------------------------------------------------------------------------------
+template <int NT, int BAR>
+__device__ __forceinline__ void group_sync() {
+  if (BAR == 0) __syncthreads();
+  else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
+}
+
+__device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int d) {
+  const uint32_t lo = __shfl_up_sync(0xffffffffu, (uint32_t)v, d);
+  const uint32_t hi = __shfl_up_sync(0xffffffffu, (uint32_t)(v >> 32), d);
+  return (uint64_t)lo | ((uint64_t)hi << 32);
+}
+
+// Exclusive prefix sum of one value per thread in rank order; *total receives the group sum.
+template <int NT, int BAR, typename T>
+__device__ __forceinline__ T group_exclusive_scan(T v, int tid, uint64_t* scratch, T* total) {
+  constexpr int NW = NT / 32;
+  const int lane = tid & 31, warp = tid >> 5;
+  T inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    T n;
+    if (sizeof(T) == 8) n = (T)shfl_up_u64((uint64_t)inc, d);
+    else n = (T)__shfl_up_sync(0xffffffffu, (uint32_t)inc, d);
+    if (lane >= d) inc += n;
+  }
+  if (lane == 31) scratch[warp] = (uint64_t)inc;
+  group_sync<NT, BAR>();
+  if (warp == 0) {
+    uint64_t w = lane < NW ? scratch[lane] : 0;
+    uint64_t winc = w;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint64_t n = shfl_up_u64(winc, d);
+      if (lane >= d) winc += n;
+    }
+    if (lane < NW) scratch[NW + lane] = winc - w;
+    if (lane == 31) scratch[2 * NW] = winc;
+  }
+  group_sync<NT, BAR>();
+  const T warp_base = (T)scratch[NW + warp];
+  *total = (T)scratch[2 * NW];
+  const T result = warp_base + inc - v;
+  group_sync<NT, BAR>();  // scratch may be reused immediately by the caller
+  return result;
+}
+
+template <int NT, int BAR>
+__device__ __forceinline__ uint64_t group_sum_u64(uint64_t v, int tid, uint64_t* scratch) {
+  constexpr int NW = NT / 32;
+  const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    const uint32_t lo = __shfl_xor_sync(0xffffffffu, (uint32_t)v, d);
+    const uint32_t hi = __shfl_xor_sync(0xffffffffu, (uint32_t)(v >> 32), d);
+    v += (uint64_t)lo | ((uint64_t)hi << 32);
+  }
+  if (lane == 0) scratch[warp] = v;
+  group_sync<NT, BAR>();
+  uint64_t t = 0;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) t += scratch[w];
+  group_sync<NT, BAR>();
+  return t;
+}
+
+template <int NT, int BAR>
+__device__ __forceinline__ float group_sum_f32(float v, int tid, uint64_t* scratch) {
+  constexpr int NW = NT / 32;
+  const int lane = tid & 31, warp = tid >> 5;
+  float* f = reinterpret_cast<float*>(scratch);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+  if (lane == 0) f[warp] = v;
+  group_sync<NT, BAR>();
+  // fixed-shape pairwise tree over the warp sums so that every thread gets the same value
+  float w = lane < NW ? f[lane] : 0.0f;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) w += __shfl_xor_sync(0xffffffffu, w, d);
+  group_sync<NT, BAR>();
+  return w;
+}
+
+template <int NT, int BAR>
+__device__ __forceinline__ float group_max_f32(float v, int tid, uint64_t* scratch) {
+  constexpr int NW = NT / 32;
+  const int lane = tid & 31, warp = tid >> 5;
+  float* f = reinterpret_cast<float*>(scratch);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, d));
+  if (lane == 0) f[warp] = v;
+  group_sync<NT, BAR>();
+  float w = lane < NW ? f[lane] : __int_as_float(0xff800000);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) w = fmaxf(w, __shfl_xor_sync(0xffffffffu, w, d));
+  group_sync<NT, BAR>();
+  return w;
+}
+
+// Fixed-point inverse-CDF draw over n entries in index order.  weight(k) returns the fixed-point
+// weight of entry k (it is evaluated twice).  Returns the selected index to every thread, or -1 when
+// the weights sum to zero.  scratch: 2*(NT/32)+4 uint64 slots.
+template <int NT, int BAR, typename WeightFn>
+__device__ __forceinline__ int group_icdf(WeightFn weight, int n, uint64_t R, int tid, uint64_t* scratch) {
+  constexpr int ITEMS = 4;
+  uint64_t local = 0;
+  for (int k = tid; k < n; k += NT) local += weight(k);
+  const uint64_t T = group_sum_u64<NT, BAR>(local, tid, scratch);
+  if (T == 0) return -1;
+  const uint64_t t = __umul64hi(R, T);
+  int* found = reinterpret_cast<int*>(scratch + 2 * (NT / 32) + 2);
+  uint64_t base = 0;
+  for (int c0 = 0; c0 < n; c0 += NT * ITEMS) {
+    const int k0 = c0 + tid * ITEMS;
+    uint64_t w[ITEMS];
+    uint64_t sum = 0;
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) {
+      w[j] = (k0 + j < n) ? weight(k0 + j) : 0ull;
+      sum += w[j];
+    }
+    uint64_t total;
+    const uint64_t lo = base + group_exclusive_scan<NT, BAR, uint64_t>(sum, tid, scratch, &total);
+    if (t >= lo && t < lo + sum) {
+      uint64_t run = lo;
+      int k = k0;
+#pragma unroll
+      for (int j = 0; j < ITEMS; ++j) {
+        run += w[j];
+        if (t < run) break;
+        ++k;
+      }
+      *found = k;
+    }
+    base += total;
+    if (t < base) break;  // uniform: every thread sees the same base
+  }
+  group_sync<NT, BAR>();
+  const int k = *found;
+  group_sync<NT, BAR>();
+  return k;
+}
+
+}  // namespace sjd

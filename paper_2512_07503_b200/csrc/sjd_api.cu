@@ -1,0 +1,162 @@
+// Host side of the C ABI declared in include/sjd.h: argument checks and kernel launches.
+// Nothing here allocates, frees or synchronises.
+#include "../../include/sjd.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+
+#include "device_utils.cuh"
+#include "row_kernels.cuh"
+#include "verify_kernel.cuh"
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+  std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+  return SJD_ERR_CUDA;
+}
+
+constexpr int kGenericThreads = 512;
+constexpr int kVerifyThreads = 256;
+
+int sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      cached = n;
+    else
+      return 148;
+  }
+  return cached;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_probs(const sjd_probs* p) {
+  if (!p || !p->tok_prob || !p->ids || !p->vals || !p->cnt) return SJD_ERR_NULL;
+  return SJD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sjd_version(void) { return SJD_VERSION; }
+
+const char* sjd_status_string(int code) {
+  switch (code) {
+    case SJD_OK: return "ok";
+    case SJD_ERR_NULL: return "a required pointer is NULL";
+    case SJD_ERR_SHAPE: return "bad shape: need B >= 0, 1 <= W <= SJD_W_MAX, V >= 8 and V % 8 == 0, top_k >= 1";
+    case SJD_ERR_ALIGN: return "logits base address or strides are not 16-byte aligned";
+    case SJD_ERR_DTYPE: return "unknown logits dtype";
+    case SJD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SJD_ERR_STRUCT: return "struct_size does not match this library";
+    case SJD_ERR_CUDA: return "CUDA runtime error";
+    case SJD_ERR_CAPACITY: return "problem exceeds the fixed capacity of this entry point";
+    default: return "unknown status";
+  }
+}
+
+const char* sjd_last_cuda_error(void) { return g_cuda_error; }
+
+size_t sjd_workspace_bytes(const sjd_params* p) {
+  if (!p || p->B < 0 || p->W < 1) return 0;
+  const size_t rows = (size_t)p->B * (size_t)p->W;
+  const size_t bytes = rows * sizeof(sjd::RowScratch) + 256;
+  return (bytes + 255) & ~(size_t)255;
+}
+
+int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* drafts, const sjd_probs* draft_probs,
+             const sjd_params* P, uint64_t philox_seed, int32_t* out_accept_len, int32_t* out_tokens,
+             sjd_probs* out_probs) {
+  if (!P) return SJD_ERR_NULL;
+  if (P->struct_size != (int32_t)sizeof(sjd_params)) return SJD_ERR_STRUCT;
+  if (!logits_cond || !out_accept_len || !out_tokens) return SJD_ERR_NULL;
+  if (check_probs(out_probs) != SJD_OK) return SJD_ERR_NULL;
+  const bool draft_all = (P->flags & SJD_FLAG_DRAFT_ALL) != 0;
+  if (!draft_all && (!drafts || check_probs(draft_probs) != SJD_OK)) return SJD_ERR_NULL;
+  if (P->B < 0 || P->W < 1 || P->W > SJD_W_MAX || P->V < 8 || (P->V % 8) != 0 || P->top_k < 1) return SJD_ERR_SHAPE;
+  if (P->logits_dtype != SJD_F32 && P->logits_dtype != SJD_BF16) return SJD_ERR_DTYPE;
+  const int64_t esize = P->logits_dtype == SJD_BF16 ? 2 : 4;
+  if (!aligned16(logits_cond) || (logits_uncond && !aligned16(logits_uncond)) || (P->stride_b * esize) % 16 != 0 ||
+      (P->stride_w * esize) % 16 != 0 || P->stride_w < P->V || P->stride_b < 0)
+    return SJD_ERR_ALIGN;
+  if (!P->workspace || (reinterpret_cast<uintptr_t>(P->workspace) & 255u) != 0 ||
+      P->workspace_bytes < sjd_workspace_bytes(P))
+    return SJD_ERR_WORKSPACE;
+  if (P->B == 0) return SJD_OK;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(P->stream);
+  const int kcap = P->top_k < P->V ? P->top_k : P->V;
+  const int rows = P->B * P->W;
+
+  sjd::RowArgs ra;
+  ra.cond = logits_cond;
+  ra.uncond = logits_uncond;
+  ra.stride_b = P->stride_b;
+  ra.stride_w = P->stride_w;
+  ra.B = P->B; ra.W = P->W; ra.V = P->V; ra.kcap = kcap;
+  ra.s = P->cfg_scale;
+  ra.inv_T = P->inv_temperature;
+  ra.win_len = P->win_len;
+  ra.pos_base = P->pos_base;
+  ra.iteration = P->iteration;
+  ra.iteration0 = P->iteration0;
+  ra.drafts = draft_all ? nullptr : drafts;
+  ra.seed_lo = (uint32_t)(philox_seed & 0xffffffffu);
+  ra.seed_hi = (uint32_t)(philox_seed >> 32);
+  ra.purpose = draft_all ? sjd::kPurposeInit : sjd::kPurposeRedraft;
+  ra.out_ids = out_probs->ids;
+  ra.out_vals = out_probs->vals;
+  ra.out_cnt = out_probs->cnt;
+  ra.scratch = static_cast<sjd::RowScratch*>(P->workspace);
+
+  {
+    const int grid = rows < 4 * sm_count() ? rows : 4 * sm_count();
+    if (P->logits_dtype == SJD_BF16)
+      sjd::rows_generic_kernel<1, kGenericThreads><<<grid, kGenericThreads, 0, stream>>>(ra);
+    else
+      sjd::rows_generic_kernel<0, kGenericThreads><<<grid, kGenericThreads, 0, stream>>>(ra);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "row kernel launch");
+  }
+
+  sjd::VerifyArgs va;
+  va.B = P->B; va.W = P->W; va.V = P->V; va.kcap = kcap;
+  va.flags = P->flags;
+  va.tau = P->reuse_tau;
+  va.win_len = P->win_len;
+  va.pos_base = P->pos_base;
+  va.iteration = P->iteration;
+  va.iteration0 = P->iteration0;
+  va.seed_lo = ra.seed_lo;
+  va.seed_hi = ra.seed_hi;
+  va.drafts = drafts;
+  va.q_tok = draft_all ? nullptr : draft_probs->tok_prob;
+  va.q_ids = draft_all ? nullptr : draft_probs->ids;
+  va.q_vals = draft_all ? nullptr : draft_probs->vals;
+  va.q_cnt = draft_all ? nullptr : draft_probs->cnt;
+  va.p_ids = out_probs->ids;
+  va.p_vals = out_probs->vals;
+  va.scratch = ra.scratch;
+  va.out_accept_len = out_accept_len;
+  va.out_tokens = out_tokens;
+  va.out_tok_prob = out_probs->tok_prob;
+  va.out_flags = P->out_flags;
+  va.status = P->status;
+  {
+    sjd::verify_kernel<kVerifyThreads><<<P->B, kVerifyThreads, 0, stream>>>(va);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "verify kernel launch");
+  }
+  return SJD_OK;
+}
+
+}  // extern "C"
