@@ -18,9 +18,10 @@
  * previous iteration.  Distributions cross the ABI in sparse form: after top-K a row has at most
  * kcap = min(top_k, V) non-zero entries, stored as ascending token ids plus probabilities.
  *
- * All arithmetic runs in the library's CUDA kernels.  The library allocates nothing, frees nothing and
- * never synchronises in sjd_step(): the caller owns every buffer, including the scratch workspace, and
- * the call returns as soon as the kernels are enqueued on params->stream.
+ * All arithmetic runs in the library's CUDA kernels.  sjd_step() allocates nothing, frees nothing and
+ * never synchronises: the caller owns every buffer, including the scratch workspace, and the call
+ * returns as soon as the kernels are enqueued on params->stream.  (The host-buffer variant at the end of
+ * this header owns device mirrors and does synchronise.)
  *
  * Random numbers: Philox4x32-10, key = (seed low word, seed high word), counter = (absolute position,
  * sequence index, Jacobi iteration, purpose); one block per decision, no state.  A uniform for the accept
@@ -53,6 +54,9 @@ extern "C" {
 #define SJD_FLAG_DRAFT_ALL 2 /* no verification: draw every valid row from its own p (initial drafts; Section
                                 4.2 strategies that sample from a predicted distribution).  accept_len = 0. */
 
+#define SJD_FLAG_FORCE_GENERIC 4 /* diagnostics: use the any-shape multi-pass row kernel even where the
+                                   single-pass streaming kernel applies (results are identical)          */
+
 /* cnt value of a row of sjd_probs that stands for the uniform distribution over V (1/V each); used for
  * window slots that were initialised at random and have no previous-iteration distribution. */
 #define SJD_Q_UNIFORM (-1)
@@ -68,6 +72,7 @@ extern "C" {
 #define SJD_STATUS_QTOK_NONPOSITIVE 1 /* q_i(x_i) <= 0 at a valid row: treated as an infinite ratio      */
 #define SJD_STATUS_EMPTY_RESIDUAL 2   /* fixed-point residual total was 0: drawn from p instead          */
 #define SJD_STATUS_DEGENERATE_ROW 4   /* a row had no finite logit: its probabilities are all 0          */
+#define SJD_STATUS_INTERNAL_TIMEOUT 8 /* a bounded on-chip wait gave up: the sequence's outputs are invalid */
 
 /* return codes */
 #define SJD_OK 0
@@ -110,6 +115,8 @@ typedef struct {
   void* workspace;            /* device scratch, 256-byte aligned, owned by the caller                     */
   size_t workspace_bytes;     /* >= sjd_workspace_bytes(params)                                            */
   void* stream;               /* cudaStream_t the work is enqueued on (NULL = legacy default stream)       */
+  void* ev_rows_begin;        /* optional cudaEvent_t recorded on `stream` just before the row stage ...   */
+  void* ev_rows_end;          /* ... and just after it (tracing; NULL = not recorded)                      */
 } sjd_params;
 
 /* Library version (SJD_VERSION of the build). */
@@ -120,6 +127,9 @@ const char* sjd_status_string(int code);
 
 /* Text of the last CUDA runtime error seen by this thread's most recent failing call ("" if none). */
 const char* sjd_last_cuda_error(void);
+
+/* Number of kernels this library has launched in this process so far (all threads, all entry points). */
+uint64_t sjd_launch_count(void);
 
 /* Scratch bytes sjd_step() needs for this shape (depends on B, W only).  0 on a NULL argument. */
 size_t sjd_workspace_bytes(const sjd_params* params);
@@ -146,6 +156,27 @@ size_t sjd_workspace_bytes(const sjd_params* params);
 int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* drafts,
              const sjd_probs* draft_probs, const sjd_params* params, uint64_t philox_seed,
              int32_t* out_accept_len, int32_t* out_tokens, sjd_probs* out_probs);
+
+/*
+ * Host-buffer variant for callers whose logits and window state live in host memory.
+ *
+ * sjd_host_ctx_create() allocates, on the current device, device copies of every argument of sjd_step()
+ * for the shape in `shape` (B, W, V, logits_dtype, top_k are read; strides are taken as contiguous
+ * [B,W,V]) plus the workspace and a stream, and returns an opaque handle.  sjd_step_host() copies the
+ * HOST arrays in (pinned memory makes the copies asynchronous and fast, pageable memory works), runs
+ * sjd_step() on the context's stream, copies every output back and returns after the stream has
+ * drained, so the host arrays are ready on return.  In `params`, B/W/V/dtype/top_k must equal the
+ * context's; win_len, pos_base, iteration, out_flags and status are HOST pointers here (or NULL);
+ * workspace, stream and the event fields are ignored.  draft_probs / out_probs hold HOST pointers.
+ * Returns SJD_OK or a negative SJD_ERR_*.  sjd_host_ctx_destroy() frees everything (NULL is allowed).
+ * A context must not be used by two threads at once.
+ */
+typedef struct sjd_host_ctx sjd_host_ctx;
+int sjd_host_ctx_create(const sjd_params* shape, sjd_host_ctx** out_ctx);
+int sjd_step_host(sjd_host_ctx* ctx, const void* logits_cond, const void* logits_uncond, const int32_t* drafts,
+                  const sjd_probs* draft_probs, const sjd_params* params, uint64_t philox_seed,
+                  int32_t* out_accept_len, int32_t* out_tokens, sjd_probs* out_probs);
+void sjd_host_ctx_destroy(sjd_host_ctx* ctx);
 
 #ifdef __cplusplus
 }

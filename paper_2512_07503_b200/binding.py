@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 SJD_F32, SJD_BF16 = 0, 1
-SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL = 1, 2
+SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL, SJD_FLAG_FORCE_GENERIC = 1, 2, 4
 SJD_Q_UNIFORM = -1
 SJD_OUT_INVALID, SJD_OUT_ACCEPTED, SJD_OUT_RESIDUAL, SJD_OUT_REUSED, SJD_OUT_RESAMPLED = 0, 1, 2, 3, 4
 SJD_STATUS_QTOK_NONPOSITIVE, SJD_STATUS_EMPTY_RESIDUAL, SJD_STATUS_DEGENERATE_ROW = 1, 2, 4
@@ -33,7 +33,8 @@ class sjd_params(C.Structure):
                 ("reuse_tau", C.c_float), ("flags", C.c_int32), ("iteration0", C.c_int32),
                 ("win_len", C.c_void_p), ("pos_base", C.c_void_p), ("iteration", C.c_void_p),
                 ("out_flags", C.c_void_p), ("status", C.c_void_p), ("workspace", C.c_void_p),
-                ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p)]
+                ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p), ("ev_rows_begin", C.c_void_p),
+                ("ev_rows_end", C.c_void_p)]
 
 
 class SjdError(RuntimeError):
@@ -53,6 +54,7 @@ def lib() -> C.CDLL:
         L.sjd_status_string.argtypes = [C.c_int]
         L.sjd_status_string.restype = C.c_char_p
         L.sjd_last_cuda_error.restype = C.c_char_p
+        L.sjd_launch_count.restype = C.c_uint64
         L.sjd_workspace_bytes.argtypes = [C.POINTER(sjd_params)]
         L.sjd_workspace_bytes.restype = C.c_size_t
         L.sjd_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs), C.POINTER(sjd_params),
@@ -64,6 +66,10 @@ def lib() -> C.CDLL:
 
 def sjd_version() -> int:
     return int(lib().sjd_version())
+
+
+def sjd_launch_count() -> int:
+    return int(lib().sjd_launch_count())
 
 
 def sjd_status_string(code: int) -> str:
@@ -151,6 +157,8 @@ def make_params(logits: torch.Tensor, *, top_k: int, cfg_scale: float = 1.0, inv
         p.workspace_bytes = workspace.numel() * workspace.element_size()
     s = stream if stream is not None else torch.cuda.current_stream(logits.device)
     p.stream = s.cuda_stream
+    # the struct only holds raw addresses: keep the tensors alive as long as the struct lives
+    p._keepalive = (win_len, pos_base, iteration, out_flags, status, workspace, s)
     return p
 
 
@@ -175,4 +183,98 @@ def sjd_step(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor], d
                               _opt_ptr(drafts), C.byref(q) if q is not None else None, C.byref(params),
                               int(philox_seed) & 0xFFFFFFFFFFFFFFFF, _opt_ptr(out_accept_len), _opt_ptr(out_tokens),
                               C.byref(o))
+    _check(code)
+
+
+# ----------------------------------------------------------------------------------------------------
+# host-buffer variant
+# ----------------------------------------------------------------------------------------------------
+@dataclass
+class HostProbs:
+    """Host (CPU, ideally pinned) arrays of one ``sjd_probs``."""
+    tok_prob: torch.Tensor
+    ids: torch.Tensor
+    vals: torch.Tensor
+    cnt: torch.Tensor
+
+    @staticmethod
+    def empty(B: int, W: int, kcap: int, pin: bool = True) -> "HostProbs":
+        mk = lambda shape, dt: torch.zeros(shape, dtype=dt, pin_memory=pin)
+        return HostProbs(mk((B, W), torch.float32), mk((B, W, kcap), torch.int32), mk((B, W, kcap), torch.float32),
+                         mk((B, W), torch.int32))
+
+    def c_struct(self) -> sjd_probs:
+        for t in (self.tok_prob, self.ids, self.vals, self.cnt):
+            if t.is_cuda or not t.is_contiguous():
+                raise SjdError("host sjd_probs arrays must be contiguous CPU tensors")
+        return sjd_probs(self.tok_prob.data_ptr(), self.ids.data_ptr(), self.vals.data_ptr(), self.cnt.data_ptr())
+
+    def nbytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in (self.tok_prob, self.ids, self.vals, self.cnt))
+
+
+def _host_ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise SjdError("host arrays must be contiguous CPU tensors")
+    return t.data_ptr()
+
+
+class HostContext:
+    """Owner of an ``sjd_host_ctx`` (device mirrors for one shape on the current device)."""
+
+    def __init__(self, B: int, W: int, V: int, logits_dtype: int, top_k: int, device=None):
+        L = lib()
+        L.sjd_host_ctx_create.argtypes = [C.POINTER(sjd_params), C.POINTER(C.c_void_p)]
+        L.sjd_host_ctx_create.restype = C.c_int
+        L.sjd_step_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs),
+                                    C.POINTER(sjd_params), C.c_uint64, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs)]
+        L.sjd_step_host.restype = C.c_int
+        L.sjd_host_ctx_destroy.argtypes = [C.c_void_p]
+        L.sjd_host_ctx_destroy.restype = None
+        self.shape = (B, W, V, logits_dtype, top_k)
+        self.device = torch.device(device if device is not None else "cuda:0")
+        p = sjd_params()
+        p.struct_size = C.sizeof(sjd_params)
+        p.B, p.W, p.V, p.logits_dtype, p.top_k = B, W, V, logits_dtype, top_k
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(L.sjd_host_ctx_create(C.byref(p), C.byref(h)))
+        self._h = h
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            with torch.cuda.device(self.device):
+                lib().sjd_host_ctx_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def params(self, *, cfg_scale=1.0, inv_temperature=1.0, reuse_tau=0.5, flags=SJD_FLAG_REUSE, iteration0=0,
+               win_len=None, pos_base=None, iteration=None, out_flags=None, status=None) -> sjd_params:
+        B, W, V, dt, top_k = self.shape
+        p = sjd_params()
+        p.struct_size = C.sizeof(sjd_params)
+        p.B, p.W, p.V, p.logits_dtype, p.top_k = B, W, V, dt, top_k
+        p.stride_b, p.stride_w = W * V, V
+        p.cfg_scale, p.inv_temperature, p.reuse_tau, p.flags, p.iteration0 = (cfg_scale, inv_temperature, reuse_tau,
+                                                                               flags, iteration0)
+        p.win_len, p.pos_base, p.iteration = _host_ptr(win_len), _host_ptr(pos_base), _host_ptr(iteration)
+        p.out_flags, p.status = _host_ptr(out_flags), _host_ptr(status)
+        return p
+
+
+def sjd_step_host(ctx: HostContext, logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor],
+                  drafts: Optional[torch.Tensor], draft_probs: Optional[HostProbs], params: sjd_params,
+                  philox_seed: int, out_accept_len: torch.Tensor, out_tokens: torch.Tensor,
+                  out_probs: HostProbs) -> None:
+    """Host-buffer step: copies in, runs the kernels, copies out; the host arrays are ready on return."""
+    q = draft_probs.c_struct() if draft_probs is not None else None
+    o = out_probs.c_struct()
+    with torch.cuda.device(ctx.device):
+        code = lib().sjd_step_host(ctx._h, _host_ptr(logits_cond), _host_ptr(logits_uncond), _host_ptr(drafts),
+                                   C.byref(q) if q is not None else None, C.byref(params),
+                                   int(philox_seed) & 0xFFFFFFFFFFFFFFFF, _host_ptr(out_accept_len),
+                                   _host_ptr(out_tokens), C.byref(o))
     _check(code)

@@ -14,6 +14,7 @@ constexpr int kPurposeRedraft = 2;
 constexpr int kPurposeInit = 3;
 
 constexpr int kRowStatusDegenerate = 1;
+constexpr int kRowStatusTimeout = 2;  // a bounded on-chip wait gave up; the row has no result
 
 // ------------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): counter = (position, sequence, iteration, purpose),
@@ -123,6 +124,22 @@ template <int NT, int BAR>
 __device__ __forceinline__ void group_sync() {
   if (BAR == 0) __syncthreads();
   else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
+}
+
+// OR of a predicate over the group (also a barrier).
+template <int NT, int BAR>
+__device__ __forceinline__ bool group_any(bool pred) {
+  if (BAR == 0) return __syncthreads_or(pred ? 1 : 0) != 0;
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, %2, %3, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)(pred ? 1 : 0)), "n"(BAR), "n"(NT)
+      : "memory");
+  return r != 0;
 }
 
 __device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int d) {

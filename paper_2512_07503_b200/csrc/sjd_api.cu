@@ -4,16 +4,21 @@
 
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 
 #include "device_utils.cuh"
 #include "row_kernels.cuh"
+#include "rows_stream.cuh"
 #include "verify_kernel.cuh"
+
+#include <cmath>
 
 namespace {
 
 thread_local char g_cuda_error[256] = "";
+std::atomic<uint64_t> g_launches{0};
 
 int cuda_fail(cudaError_t e, const char* what) {
   std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", what, cudaGetErrorString(e));
@@ -34,6 +39,57 @@ int sm_count() {
       return 148;
   }
   return cached;
+}
+
+constexpr int kStreamConsumerWarps = 16;
+constexpr int kStreamStages = 3;
+
+// Decide whether the single-pass streaming kernel can take this shape, and with which sampling
+// parameters.  The sample is every SS-th 256-element tile of a row; its rank-m value (from the top)
+// becomes the candidate threshold.  m is chosen six standard deviations above K/SS, so that a row with
+// exchangeable entries fails to deliver K candidates with probability below 1e-9 (such a row is redone
+// by the generic path, never answered wrongly).
+bool plan_stream(const sjd_params* P, int kcap, sjd::StreamCfg* cfg, size_t* smem) {
+  const int V = P->V;
+  const int tps = P->logits_dtype == SJD_BF16 ? 32 : 16;
+  if (kcap > sjd::kStageKcapMax || V % sjd::kTileElems != 0) return false;
+  const int tiles = V / sjd::kTileElems;
+  int ss = 0;
+  for (int cand : {8, 16, 32}) {
+    if (tiles % cand == 0 && tiles / cand <= tps) {
+      ss = cand;
+      break;
+    }
+  }
+  if (ss == 0) return false;
+  const int n_sample = V / ss;
+  const double a = (double)kcap / ss;
+  const double root = 3.0 + std::sqrt(9.0 + a);
+  const int m = (int)std::ceil(root * root);
+  if (m > n_sample / 2) return false;
+  // expected candidates, six sigma above, must fit the per-thread lists with room to spare
+  const double expect = ((double)m + 6.0 * std::sqrt((double)m)) * ss * 1.25;
+  const int nt = kStreamConsumerWarps * 32;
+  if (expect > 0.75 * (double)sjd::kLaneListCap * nt) return false;
+  cfg->sample_stride = ss;
+  cfg->sample_rank = m;
+  cfg->n_stages = kStreamStages;
+  cfg->vwords = V / 32;
+  *smem = sjd::stream_smem_bytes(cfg->n_stages, nt, cfg->vwords);
+  return *smem <= 227u * 1024u;
+}
+
+template <int DTYPE>
+cudaError_t launch_stream(const sjd::RowArgs& ra, const sjd::StreamCfg& cfg, size_t smem, int grid, cudaStream_t st) {
+  auto kern = sjd::rows_stream_kernel<DTYPE, kStreamConsumerWarps>;
+  static bool configured = false;  // per instantiation; the attribute is sticky for the process
+  if (!configured) {
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  kern<<<grid, kStreamConsumerWarps * 32 + 32, smem, st>>>(ra, cfg);
+  return cudaGetLastError();
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -65,6 +121,8 @@ const char* sjd_status_string(int code) {
 }
 
 const char* sjd_last_cuda_error(void) { return g_cuda_error; }
+
+uint64_t sjd_launch_count(void) { return g_launches.load(); }
 
 size_t sjd_workspace_bytes(const sjd_params* p) {
   if (!p || p->B < 0 || p->W < 1) return 0;
@@ -118,14 +176,32 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
   ra.out_cnt = out_probs->cnt;
   ra.scratch = static_cast<sjd::RowScratch*>(P->workspace);
 
+  if (P->ev_rows_begin) {
+    const cudaError_t e = cudaEventRecord(static_cast<cudaEvent_t>(P->ev_rows_begin), stream);
+    if (e != cudaSuccess) return cuda_fail(e, "event record");
+  }
   {
-    const int grid = rows < 4 * sm_count() ? rows : 4 * sm_count();
-    if (P->logits_dtype == SJD_BF16)
-      sjd::rows_generic_kernel<1, kGenericThreads><<<grid, kGenericThreads, 0, stream>>>(ra);
-    else
-      sjd::rows_generic_kernel<0, kGenericThreads><<<grid, kGenericThreads, 0, stream>>>(ra);
-    const cudaError_t e = cudaGetLastError();
+    sjd::StreamCfg cfg;
+    size_t smem = 0;
+    cudaError_t e;
+    if (!(P->flags & SJD_FLAG_FORCE_GENERIC) && plan_stream(P, kcap, &cfg, &smem)) {
+      const int grid = rows < sm_count() ? rows : sm_count();
+      e = P->logits_dtype == SJD_BF16 ? launch_stream<1>(ra, cfg, smem, grid, stream)
+                                      : launch_stream<0>(ra, cfg, smem, grid, stream);
+    } else {
+      const int grid = rows < 4 * sm_count() ? rows : 4 * sm_count();
+      if (P->logits_dtype == SJD_BF16)
+        sjd::rows_generic_kernel<1, kGenericThreads><<<grid, kGenericThreads, 0, stream>>>(ra);
+      else
+        sjd::rows_generic_kernel<0, kGenericThreads><<<grid, kGenericThreads, 0, stream>>>(ra);
+      e = cudaGetLastError();
+    }
     if (e != cudaSuccess) return cuda_fail(e, "row kernel launch");
+    ++g_launches;
+  }
+  if (P->ev_rows_end) {
+    const cudaError_t e = cudaEventRecord(static_cast<cudaEvent_t>(P->ev_rows_end), stream);
+    if (e != cudaSuccess) return cuda_fail(e, "event record");
   }
 
   sjd::VerifyArgs va;
@@ -155,6 +231,7 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
     sjd::verify_kernel<kVerifyThreads><<<P->B, kVerifyThreads, 0, stream>>>(va);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "verify kernel launch");
+    ++g_launches;
   }
   return SJD_OK;
 }
