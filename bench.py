@@ -152,7 +152,7 @@ def device_inputs(wl, device, seed):
 class DeviceSet:
     """One input set on the device with its outputs and parameters."""
 
-    def __init__(self, sjd, wl, device, seed):
+    def __init__(self, sjd, wl, device, seed, seq_base=0):
         import torch
         self.wl = wl
         cond, uncond, prev_c, prev_u, self.win_len, self.pos_base = device_inputs(wl, device, seed)
@@ -167,7 +167,7 @@ class DeviceSet:
         self.status = torch.zeros(B, dtype=torch.int32, device=device)
         common = dict(top_k=wl.top_k, cfg_scale=wl.cfg_scale, inv_temperature=float(wl.inv_temperature),
                       reuse_tau=wl.reuse_tau, win_len=self.win_len, pos_base=self.pos_base, out_flags=self.flags,
-                      status=self.status)
+                      status=self.status, seq_base=seq_base)
         p0 = sjd.make_params(cond, flags=sjd.binding.SJD_FLAG_DRAFT_ALL, iteration0=0, **common)
         self.ws = torch.empty(sjd.sjd_workspace_bytes(p0), dtype=torch.uint8, device=device)
         p0.workspace, p0.workspace_bytes = self.ws.data_ptr(), self.ws.numel()
@@ -189,6 +189,7 @@ def run_ours(args):
     import torch.distributed as dist
 
     import paper_2512_07503_b200 as sjd
+    from paper_2512_07503_b200 import sharding
     from paper_2512_07503_b200 import workloads as wk
 
     if not torch.cuda.is_available():
@@ -203,7 +204,9 @@ def run_ours(args):
     wl = wk.CONFIGS[args.workload]
     K, Wm = args.steps, max(args.warmup, 3)
 
-    sets = [DeviceSet(sjd, wl, device, wl.seed + 1000 * rank + j) for j in range(NBUF)]
+    # every rank owns wl.B sequences of a global batch of world * wl.B (weak scaling over sequences)
+    seq_lo, _ = sharding.shard_range(world * wl.B, rank, world)
+    sets = [DeviceSet(sjd, wl, device, wl.seed + 1000 * rank + j, seq_base=seq_lo) for j in range(NBUF)]
     tokens_per_step = int(sum(int(s.win_len.sum().item()) for s in sets) / NBUF)
 
     def barrier():
@@ -249,10 +252,7 @@ def run_ours(args):
     if sampler:
         clocks = sampler.stop()
 
-    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    elapsed_ms = float(t.item())
+    elapsed_ms = sharding.max_over_ranks(elapsed_ms, device)
     ms_per_step = elapsed_ms / K
     value = world * tokens_per_step * K / (elapsed_ms * 1e-3)
 

@@ -107,6 +107,8 @@ typedef struct {
   float reuse_tau;            /* tau of Eq. reuse (the paper uses 0.5)                                     */
   int32_t flags;              /* SJD_FLAG_*                                                                */
   int32_t iteration0;         /* Jacobi iteration index used when `iteration` is NULL                      */
+  int32_t seq_base;           /* global index of sequence 0 of this call: the generator's sequence word is
+                                 seq_base + b, so a batch split over calls or GPUs draws the same numbers  */
   const int32_t* win_len;     /* [B] device, valid rows per sequence (ragged windows); NULL = W            */
   const int32_t* pos_base;    /* [B] device, absolute image-token index of window row 0; NULL = 0          */
   const int32_t* iteration;   /* [B] device, per-sequence iteration index; NULL = iteration0               */

@@ -47,7 +47,7 @@ class _Params(C.Structure):
                 ("stride_b", C.c_int64), ("stride_w", C.c_int64), ("cfg_scale", C.c_float),
                 ("inv_temperature", C.c_float), ("top_k", C.c_int32), ("reuse_tau", C.c_float),
                 ("flags", C.c_int32), ("win_len", C.c_void_p), ("pos_base", C.c_void_p),
-                ("iteration", C.c_void_p), ("iteration0", C.c_int32), ("n_threads", C.c_int32)]
+                ("iteration", C.c_void_p), ("iteration0", C.c_int32), ("n_threads", C.c_int32), ("seq_base", C.c_int32)]
 
 
 class _Diag(C.Structure):
@@ -199,7 +199,7 @@ _DIAG_I = ("pot_ok", "pot_reuse", "pot_redraft", "pot_residual")
 
 def sjd_step(logits_cond, logits_uncond, drafts, draft_probs, *, dtype, V, cfg_scale=1.0, inv_temperature=1.0,
              top_k, reuse_tau=0.5, flags=FLAG_REUSE, win_len=None, pos_base=None, iteration=None, iteration0=0,
-             seed=0, n_threads=1, diag=False) -> StepResult:
+             seed=0, n_threads=1, diag=False, seq_base=0) -> StepResult:
     """One verify-and-redraft step on host arrays shaped [B,W,V] (contiguous)."""
     cond = _logits_view(logits_cond, dtype)
     unc = _logits_view(logits_uncond, dtype)
@@ -221,7 +221,7 @@ def sjd_step(logits_cond, logits_uncond, drafts, draft_probs, *, dtype, V, cfg_s
         return a.ctypes.data
 
     P = _Params(B, W, V, dtype, W * V, V, cfg_scale, inv_temperature, top_k, reuse_tau, flags, opt_i32(win_len),
-                opt_i32(pos_base), opt_i32(iteration), iteration0, n_threads)
+                opt_i32(pos_base), opt_i32(iteration), iteration0, n_threads, seq_base)
     d = {}
     dstruct = None
     if diag:

@@ -209,6 +209,7 @@ void verify_phase(const StepCtx& c, int32_t b, const std::vector<int32_t>& degen
   const int32_t W = P.W, V = P.V, L = seq_len(c, b);
   const int32_t pos0 = P.pos_base ? P.pos_base[b] : 0;
   const int32_t iter = P.iteration ? P.iteration[b] : P.iteration0;
+  const int32_t gb = P.seq_base + b;  // sequence word of the counter
   const bool draft_all = (P.flags & ORC_FLAG_DRAFT_ALL) != 0;
   const bool reuse_on = (P.flags & ORC_FLAG_REUSE) != 0;
   int32_t st = 0;
@@ -229,7 +230,7 @@ void verify_phase(const StepCtx& c, int32_t b, const std::vector<int32_t>& degen
       const int32_t tok = c.drafts[r];
       const float qt = c.q->tok_prob[r];
       ptok[(size_t)i] = lookup(ids, vals, cnt, V, tok);
-      draw(c.seed, pos0 + i, b, iter, ORC_PURPOSE_ACCEPT, x);
+      draw(c.seed, pos0 + i, gb, iter, ORC_PURPOSE_ACCEPT, x);
       const float u = uniform24(x[0]);
       if (!(qt > 0.0f)) st |= ORC_STATUS_QTOK_NONPOSITIVE;
       ok[(size_t)i] = accept(ptok[(size_t)i], qt, u, &ratio[(size_t)i]);
@@ -247,7 +248,7 @@ void verify_phase(const StepCtx& c, int32_t b, const std::vector<int32_t>& degen
     }
     // what the row would get if resampled from its current distribution (Eq. reuse, second case;
     // Eq. refine-sjd); evaluated for every row because the draw depends only on the row's counter
-    draw(c.seed, pos0 + i, b, iter, draft_all ? ORC_PURPOSE_INIT : ORC_PURPOSE_REDRAFT, x);
+    draw(c.seed, pos0 + i, gb, iter, draft_all ? ORC_PURPOSE_INIT : ORC_PURPOSE_REDRAFT, x);
     float mg = 0.f;
     int32_t k = icdf(vals, cnt, r64(x), &mg);
     if (k < 0) k = 0;
@@ -268,7 +269,7 @@ void verify_phase(const StepCtx& c, int32_t b, const std::vector<int32_t>& degen
     std::vector<float> w((size_t)cnt);
     residual_weights(ids, vals, cnt, c.q->ids + r * c.kcap, c.q->vals + r * c.kcap, c.q->cnt[r], V, w.data());
     uint32_t x[4];
-    draw(c.seed, pos0 + i, b, iter, ORC_PURPOSE_RESIDUAL, x);
+    draw(c.seed, pos0 + i, gb, iter, ORC_PURPOSE_RESIDUAL, x);
     int32_t k = icdf(w.data(), cnt, r64(x), margin);
     *empty = false;
     if (k < 0) {  // analytically impossible after a rejection; rounding can produce it

@@ -79,6 +79,9 @@ typedef struct {
   const int32_t* iteration; /* [B] Jacobi iteration index, NULL = iteration0                  */
   int32_t iteration0;
   int32_t n_threads;        /* rows are split over this many std::thread workers (>=1)        */
+  int32_t seq_base;         /* global index of sequence 0 of this call: the Philox counter's
+                               sequence word is seq_base + b (a batch split over several
+                               calls or devices draws the same numbers as the whole batch)   */
 } orc_params;
 
 /* Optional per-position diagnostics (any pointer may be NULL).  "Potential" outcomes are

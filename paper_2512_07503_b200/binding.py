@@ -30,7 +30,7 @@ class sjd_params(C.Structure):
     _fields_ = [("struct_size", C.c_int32), ("B", C.c_int32), ("W", C.c_int32), ("V", C.c_int32),
                 ("logits_dtype", C.c_int32), ("stride_b", C.c_int64), ("stride_w", C.c_int64),
                 ("cfg_scale", C.c_float), ("inv_temperature", C.c_float), ("top_k", C.c_int32),
-                ("reuse_tau", C.c_float), ("flags", C.c_int32), ("iteration0", C.c_int32),
+                ("reuse_tau", C.c_float), ("flags", C.c_int32), ("iteration0", C.c_int32), ("seq_base", C.c_int32),
                 ("win_len", C.c_void_p), ("pos_base", C.c_void_p), ("iteration", C.c_void_p),
                 ("out_flags", C.c_void_p), ("status", C.c_void_p), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p), ("ev_rows_begin", C.c_void_p),
@@ -125,7 +125,7 @@ def make_params(logits: torch.Tensor, *, top_k: int, cfg_scale: float = 1.0, inv
                 win_len: Optional[torch.Tensor] = None, pos_base: Optional[torch.Tensor] = None,
                 iteration: Optional[torch.Tensor] = None, out_flags: Optional[torch.Tensor] = None,
                 status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-                stream: Optional[torch.cuda.Stream] = None) -> sjd_params:
+                stream: Optional[torch.cuda.Stream] = None, seq_base: int = 0) -> sjd_params:
     """Fill an ``sjd_params`` from a [B,W,V] logits tensor (fp32 or bf16, vocabulary axis contiguous)."""
     if logits.dim() != 3 or logits.stride(2) != 1:
         raise SjdError("logits must be [B,W,V] with a contiguous vocabulary axis")
@@ -147,6 +147,7 @@ def make_params(logits: torch.Tensor, *, top_k: int, cfg_scale: float = 1.0, inv
     p.reuse_tau = reuse_tau
     p.flags = flags
     p.iteration0 = iteration0
+    p.seq_base = seq_base
     p.win_len = _opt_ptr(win_len)
     p.pos_base = _opt_ptr(pos_base)
     p.iteration = _opt_ptr(iteration)
@@ -252,7 +253,7 @@ class HostContext:
     __del__ = close
 
     def params(self, *, cfg_scale=1.0, inv_temperature=1.0, reuse_tau=0.5, flags=SJD_FLAG_REUSE, iteration0=0,
-               win_len=None, pos_base=None, iteration=None, out_flags=None, status=None) -> sjd_params:
+               win_len=None, pos_base=None, iteration=None, out_flags=None, status=None, seq_base=0) -> sjd_params:
         B, W, V, dt, top_k = self.shape
         p = sjd_params()
         p.struct_size = C.sizeof(sjd_params)
@@ -260,6 +261,7 @@ class HostContext:
         p.stride_b, p.stride_w = W * V, V
         p.cfg_scale, p.inv_temperature, p.reuse_tau, p.flags, p.iteration0 = (cfg_scale, inv_temperature, reuse_tau,
                                                                                flags, iteration0)
+        p.seq_base = seq_base
         p.win_len, p.pos_base, p.iteration = _host_ptr(win_len), _host_ptr(pos_base), _host_ptr(iteration)
         p.out_flags, p.status = _host_ptr(out_flags), _host_ptr(status)
         return p

@@ -28,6 +28,7 @@ struct RowArgs {
   const int32_t* pos_base;
   const int32_t* iteration;
   int iteration0;
+  int seq_base;  // global index of sequence 0 (sequence word of the generator's counter)
   const int32_t* drafts;  // nullptr when every row is drafted
   uint32_t seed_lo, seed_hi;
   int purpose;  // kPurposeRedraft or kPurposeInit
@@ -181,7 +182,7 @@ __device__ void row_generic(const RowArgs& a, int row, int tid, GenericSmem& sm)
   // ---- the row's own draw from p_i ----
   const int pos = (a.pos_base ? a.pos_base[b] : 0) + i;
   const int iter = a.iteration ? a.iteration[b] : a.iteration0;
-  const Philox4 rnd = philox4x32_10((uint32_t)pos, (uint32_t)b, (uint32_t)iter, (uint32_t)a.purpose, a.seed_lo,
+  const Philox4 rnd = philox4x32_10((uint32_t)pos, (uint32_t)(a.seq_base + b), (uint32_t)iter, (uint32_t)a.purpose, a.seed_lo,
                                     a.seed_hi);
   int k = group_icdf<NT, BAR>([&](int kk) { return fixed_weight(vals[kk]); }, kcap, random64(rnd), tid, sm.scan);
   if (k < 0) k = 0;

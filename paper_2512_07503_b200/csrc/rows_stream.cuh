@@ -597,7 +597,7 @@ __global__ void __launch_bounds__(NCW * 32 + 32, 1) rows_stream_kernel(const Row
     const int pos = (a.pos_base ? a.pos_base[b] : 0) + i;
     const int iter = a.iteration ? a.iteration[b] : a.iteration0;
     const Philox4 rnd =
-        philox4x32_10((uint32_t)pos, (uint32_t)b, (uint32_t)iter, (uint32_t)a.purpose, a.seed_lo, a.seed_hi);
+        philox4x32_10((uint32_t)pos, (uint32_t)(a.seq_base + b), (uint32_t)iter, (uint32_t)a.purpose, a.seed_lo, a.seed_hi);
     int k = group_icdf<NT, BAR>([&](int kk) { return fixed_weight(sm.st_vals[kk]); }, kcap, random64(rnd), tid, sm.scan);
     if (k < 0) k = 0;
     if (tid == 0) {

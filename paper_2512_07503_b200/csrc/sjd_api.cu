@@ -167,6 +167,7 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
   ra.pos_base = P->pos_base;
   ra.iteration = P->iteration;
   ra.iteration0 = P->iteration0;
+  ra.seq_base = P->seq_base;
   ra.drafts = draft_all ? nullptr : drafts;
   ra.seed_lo = (uint32_t)(philox_seed & 0xffffffffu);
   ra.seed_hi = (uint32_t)(philox_seed >> 32);
@@ -212,6 +213,7 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
   va.pos_base = P->pos_base;
   va.iteration = P->iteration;
   va.iteration0 = P->iteration0;
+  va.seq_base = P->seq_base;
   va.seed_lo = ra.seed_lo;
   va.seed_hi = ra.seed_hi;
   va.drafts = drafts;

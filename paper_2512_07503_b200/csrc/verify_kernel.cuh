@@ -24,6 +24,7 @@ struct VerifyArgs {
   const int32_t* pos_base;
   const int32_t* iteration;
   int iteration0;
+  int seq_base;
   uint32_t seed_lo, seed_hi;
   const int32_t* drafts;
   // previous-iteration distributions
@@ -98,7 +99,7 @@ __device__ void verify_sequence(const VerifyArgs& a, int b, int tid, VerifySmem&
     if (!draft_all) {
       const float q = a.q_tok[base + i];
       const float ratio = likelihood_ratio(rs.p_tok, q);
-      const Philox4 rnd = philox4x32_10((uint32_t)(pos0 + i), (uint32_t)b, (uint32_t)iter, kPurposeAccept, a.seed_lo,
+      const Philox4 rnd = philox4x32_10((uint32_t)(pos0 + i), (uint32_t)(a.seq_base + b), (uint32_t)iter, kPurposeAccept, a.seed_lo,
                                         a.seed_hi);
       const float u = uniform24(rnd.x0);
       if (!(u < fminf(ratio, 1.0f))) atomicMin(&sm.first_reject, i);
@@ -118,7 +119,7 @@ __device__ void verify_sequence(const VerifyArgs& a, int b, int tid, VerifySmem&
     const float* qv = a.q_vals + r * a.kcap;
     const int qc = a.q_cnt[r];
     const float q_uniform = __fdiv_rn(1.0f, (float)a.V);
-    const Philox4 rnd = philox4x32_10((uint32_t)(pos0 + acc), (uint32_t)b, (uint32_t)iter, kPurposeResidual,
+    const Philox4 rnd = philox4x32_10((uint32_t)(pos0 + acc), (uint32_t)(a.seq_base + b), (uint32_t)iter, kPurposeResidual,
                                       a.seed_lo, a.seed_hi);
     auto residual = [&](int k) {
       const float q = (qc == kQUniform) ? q_uniform : sparse_lookup(qid, qv, qc, pid[k]);
