@@ -1,0 +1,865 @@
+// Pipelined row kernel: the sampling head (guidance merge, temperature, top-K, softmax, per-row draw) in
+// ONE pass over the logits, with the three parts of the work running concurrently on every SM.
+//
+// Persistent CTAs, one per SM, rows round-robin.  Three roles inside a CTA:
+//
+//   producer (1 warp)   streams each row through a ring of shared-memory stages with bulk asynchronous
+//                       copies (cp.async.bulk, completion on mbarriers; no multicast, own CTA only).
+//   filter (NF warps)   turns the staged bf16/fp32 pairs into merged logits y and keeps only the few per
+//                       cent that can still be in the top-K.  The first stages of a row are a strided
+//                       SAMPLE of it (every SS-th 256-element tile); a two-level histogram of the
+//                       sample's order-preserving keys gives the threshold tau0 whose rank in the sample
+//                       is high enough that at least K elements of the row reach it (a row for which
+//                       that fails is redone exactly, see below).  Every element with y >= tau0 is
+//                       appended to the warp's candidate list in shared memory.
+//   finisher (NP warps) works on the PREVIOUS row's candidates while the filter streams the next row:
+//                       exact K-th largest (linear-bin histogram + ranking inside the threshold bin,
+//                       ties to the lower id), ascending-id order through a bitmap over token ids,
+//                       softmax, coalesced output, and the row's own inverse-CDF draw.
+//
+// Candidate lists are double buffered; filter and finisher hand them over through two mbarrier pairs.
+// A row whose candidates do not contain the top-K for sure (fewer than K of them) or do not fit the
+// on-chip capacities is redone by row_generic() from global memory: the result is exact for any input.
+//
+// Every wait on an mbarrier is bounded (poll count and clock); on a time-out the CTA marks its
+// remaining rows with kRowStatusTimeout, drains its own copies in flight and returns.
+#pragma once
+
+#include "device_utils.cuh"
+#include "row_kernels.cuh"
+
+namespace sjd {
+
+constexpr int kTileElems = 256;           // elements per tile: one warp iteration, 8 per lane
+constexpr int kStageArrayBytes = 8192;    // bytes of ONE logits array in a ring stage
+constexpr int kCoarseBins = 2048;         // sample histogram, level 1: key >> 21
+constexpr int kFineBins = 256;            // sample histogram, level 2: (key >> 13) & 0xff inside one coarse bin
+constexpr int kSelBins = 2048;            // finisher's linear bins over [tau0, max]
+constexpr int kWarpListCap = 512;         // candidates one filter warp can hold for a row
+constexpr int kBinListCap = 512;          // members of the threshold bin ranked by brute force
+constexpr int kKcapMax = 2048;            // largest kcap the on-chip path stages
+constexpr int kFinItems = 8;              // staged entries per finisher thread (kKcapMax / finisher threads)
+constexpr uint32_t kSpinLimit = 1u << 22; // polls before a wait gives up
+constexpr long long kSpinCycles = 1ll << 31;  // ... or this many clock cycles, whichever comes first
+
+struct PipeCfg {
+  int sample_stride;  // SS: every SS-th tile of a row is a sample tile
+  int sample_rank;    // m: rank (from the top) within the sample that fixes tau0
+  int n_stages;       // ring depth
+  int vwords;         // V / 32
+};
+
+struct Candidate {
+  float y;
+  int32_t id;
+};
+
+// ---------------------------------------------------------------------------------------------------
+// PTX wrappers: mbarrier, 1-D bulk copy global -> shared, packed fp32 pairs
+// ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the phase did not complete within kSpinLimit polls or kSpinCycles clocks.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && clock64() - t0 > kSpinCycles) break;
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+
+// Two fp32 values in one 64-bit register; each half of a packed operation is rounded exactly like the
+// scalar operation (round to nearest even, no flush to zero).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+// max of three; a NaN operand is ignored
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Row schedule shared by the producer and the filter.
+// Tiles of a row: g = 0 .. V/256-1.  Sample tiles: g % SS == 0.  The first `sample_stages` stages hold
+// the sample tiles in order; the others hold the tail tiles t = 0.. in order, where tail tile t is
+// global tile (t/(SS-1)) SS + 1 + t%(SS-1).
+// ---------------------------------------------------------------------------------------------------
+struct RowSchedule {
+  int tiles, ss, sample_tiles, tail_tiles, sample_stages, stages;
+  __device__ __forceinline__ RowSchedule(int V, int SS, int TPS) {
+    ss = SS;
+    tiles = V / kTileElems;
+    sample_tiles = tiles / SS;
+    tail_tiles = tiles - sample_tiles;
+    sample_stages = (sample_tiles + TPS - 1) / TPS;
+    stages = sample_stages + (tail_tiles + TPS - 1) / TPS;
+  }
+  __device__ __forceinline__ int stage_tiles(int s, int TPS) const {
+    return s < sample_stages ? min(TPS, sample_tiles - TPS * s) : min(TPS, tail_tiles - TPS * (s - sample_stages));
+  }
+  __device__ __forceinline__ int global_tile(int s, int j, int TPS) const {
+    if (s < sample_stages) return (s * TPS + j) * ss;
+    const int t = TPS * (s - sample_stages) + j;
+    const int run = t / (ss - 1);
+    return run * ss + 1 + (t - run * (ss - 1));
+  }
+};
+
+template <int DTYPE>
+struct PipeTraits {
+  static constexpr int kElemBytes = DTYPE == 1 ? 2 : 4;
+  static constexpr int kTileBytes = kTileElems * kElemBytes;
+  static constexpr int kTilesPerStage = kStageArrayBytes / kTileBytes;  // 16 (bf16) or 8 (fp32)
+  static constexpr int kStageBytes = 2 * kStageArrayBytes;
+};
+
+// Element index inside a tile of the j-th value a lane holds.  bf16: 8 consecutive elements per lane
+// (one 16-byte load).  fp32: elements 4*lane..+3 and 128+4*lane..+3 (two conflict-free 16-byte loads).
+template <int DTYPE>
+__device__ __forceinline__ int tile_elem(int lane, int j) {
+  if (DTYPE == 1) return lane * 8 + j;
+  return j < 4 ? lane * 4 + j : 128 + lane * 4 + (j - 4);
+}
+
+// Merged logits y of the lane's eight elements of a staged tile, as four packed pairs:
+// d = c - u; g = fma(s, d, u); y = g * inv_T, one rounding per operation.  Multiplying by 1.0f is exact,
+// so the last step is skipped when inv_T == 1.
+template <int DTYPE>
+__device__ __forceinline__ void tile_y8(const unsigned char* ctile, const unsigned char* utile, bool has_u, bool has_t,
+                                        int lane, uint64_t s2, uint64_t t2, float (&y)[8]) {
+  uint64_t c[4], u[4];
+  if (DTYPE == 1) {
+    const uint4 w = *reinterpret_cast<const uint4*>(ctile + lane * 16);
+    c[0] = pack2(bf16_lo(w.x), bf16_hi(w.x)); c[1] = pack2(bf16_lo(w.y), bf16_hi(w.y));
+    c[2] = pack2(bf16_lo(w.z), bf16_hi(w.z)); c[3] = pack2(bf16_lo(w.w), bf16_hi(w.w));
+    if (has_u) {
+      const uint4 v = *reinterpret_cast<const uint4*>(utile + lane * 16);
+      u[0] = pack2(bf16_lo(v.x), bf16_hi(v.x)); u[1] = pack2(bf16_lo(v.y), bf16_hi(v.y));
+      u[2] = pack2(bf16_lo(v.z), bf16_hi(v.z)); u[3] = pack2(bf16_lo(v.w), bf16_hi(v.w));
+    }
+  } else {
+    const float4 a = *reinterpret_cast<const float4*>(ctile + lane * 16);
+    const float4 b = *reinterpret_cast<const float4*>(ctile + 512 + lane * 16);
+    c[0] = pack2(a.x, a.y); c[1] = pack2(a.z, a.w); c[2] = pack2(b.x, b.y); c[3] = pack2(b.z, b.w);
+    if (has_u) {
+      const float4 p = *reinterpret_cast<const float4*>(utile + lane * 16);
+      const float4 q = *reinterpret_cast<const float4*>(utile + 512 + lane * 16);
+      u[0] = pack2(p.x, p.y); u[1] = pack2(p.z, p.w); u[2] = pack2(q.x, q.y); u[3] = pack2(q.z, q.w);
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    uint64_t g = c[k];
+    if (has_u) g = fma2(s2, sub2(c[k], u[k]), u[k]);
+    if (has_t) g = mul2(g, t2);
+    unpack2(g, y[2 * k], y[2 * k + 1]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Shared-memory layout (dynamic)
+// ---------------------------------------------------------------------------------------------------
+enum {
+  kCtlAbort = 0,      // a bounded wait gave up somewhere in this CTA
+  kCtlFBin, kCtlFAbove, kCtlFCount, kCtlTau0,          // filter group
+  kCtlPBin, kCtlPAbove, kCtlPCount, kCtlGather,        // finisher group
+  kCtlPtok, kCtlFoundId, kCtlFoundP,
+  kCtlWords = 16
+};
+
+struct RowMeta {      // what the filter tells the finisher about a row, one per candidate buffer
+  float tau0;
+  float vmax[16];     // per filter warp: largest y of the tiles it saw
+  int count[16];      // per filter warp: candidates appended (may exceed kWarpListCap: overflow)
+};
+
+template <int NF>
+struct PipeSmem {
+  uint64_t* full;       // [n_stages]  ring: data landed
+  uint64_t* empty;      // [n_stages]  ring: all filter warps done with the stage
+  uint64_t* cand_full;  // [2]         candidate buffer handed to the finisher
+  uint64_t* cand_free;  // [2]         candidate buffer handed back
+  unsigned char* ring;  // [n_stages][2][kStageArrayBytes]
+  Candidate* lists;     // [2][NF][kWarpListCap]
+  RowMeta* meta;        // [2]
+  uint32_t* coarse;     // [kCoarseBins]   (filter)
+  uint32_t* fine;       // [kFineBins]     (filter)
+  uint32_t* sel;        // [kSelBins]      (finisher)
+  uint32_t* bitmap;     // [vwords]        (finisher)
+  uint16_t* wprefix;    // [vwords]        (finisher)
+  Candidate* binlist;   // [kBinListCap]   (finisher)
+  int32_t* st_ids;      // [kKcapMax]      (finisher)
+  float* st_vals;       // [kKcapMax]      (finisher)
+  uint64_t* scan_f;     // group scratch, filter
+  uint64_t* scan_p;     // group scratch, finisher
+  int* ctl;             // control words
+};
+
+__host__ __device__ inline size_t pipe_smem_fixed_bytes(int NF, int vwords) {
+  size_t b = 0;
+  b += 32 * 8;                                          // mbarriers (2 per ring stage + 4)
+  b += (size_t)2 * NF * kWarpListCap * sizeof(Candidate);
+  b += 2 * sizeof(RowMeta);
+  b += (size_t)(kCoarseBins + kFineBins + kSelBins) * 4;
+  b += (size_t)vwords * 4 + (size_t)vwords * 2;
+  b += (size_t)kBinListCap * sizeof(Candidate);
+  b += (size_t)kKcapMax * 8;
+  b += 2 * (2 * 32 + 8) * 8;
+  b += kCtlWords * 4;
+  return b + 128;  // alignment slack
+}
+__host__ __device__ inline size_t pipe_smem_bytes(int n_stages, int NF, int vwords) {
+  return pipe_smem_fixed_bytes(NF, vwords) + (size_t)n_stages * 2 * kStageArrayBytes;
+}
+
+template <int NF>
+__device__ __forceinline__ PipeSmem<NF> carve_pipe_smem(unsigned char* base, int n_stages, int vwords) {
+  PipeSmem<NF> s;
+  uintptr_t p = (reinterpret_cast<uintptr_t>(base) + 127) & ~(uintptr_t)127;
+  s.ring = reinterpret_cast<unsigned char*>(p);
+  p += (size_t)n_stages * 2 * kStageArrayBytes;
+  s.lists = reinterpret_cast<Candidate*>(p);
+  p += (size_t)2 * NF * kWarpListCap * sizeof(Candidate);
+  s.st_ids = reinterpret_cast<int32_t*>(p);
+  p += (size_t)kKcapMax * 4;
+  s.st_vals = reinterpret_cast<float*>(p);
+  p += (size_t)kKcapMax * 4;
+  s.coarse = reinterpret_cast<uint32_t*>(p);
+  p += (size_t)kCoarseBins * 4;
+  s.fine = reinterpret_cast<uint32_t*>(p);
+  p += (size_t)kFineBins * 4;
+  s.sel = reinterpret_cast<uint32_t*>(p);
+  p += (size_t)kSelBins * 4;
+  s.bitmap = reinterpret_cast<uint32_t*>(p);
+  p += (size_t)vwords * 4;
+  s.binlist = reinterpret_cast<Candidate*>(p);
+  p += (size_t)kBinListCap * sizeof(Candidate);
+  s.full = reinterpret_cast<uint64_t*>(p);
+  s.empty = s.full + n_stages;
+  s.cand_full = s.empty + n_stages;
+  s.cand_free = s.cand_full + 2;
+  p += 32 * 8;
+  s.scan_f = reinterpret_cast<uint64_t*>(p);
+  p += (2 * 32 + 8) * 8;
+  s.scan_p = reinterpret_cast<uint64_t*>(p);
+  p += (2 * 32 + 8) * 8;
+  s.meta = reinterpret_cast<RowMeta*>(p);
+  p += 2 * sizeof(RowMeta);
+  s.ctl = reinterpret_cast<int*>(p);
+  p += kCtlWords * 4;
+  s.wprefix = reinterpret_cast<uint16_t*>(p);
+  return s;
+}
+
+// Largest bin b with (entries in bins > b) < target <= (entries in bins >= b).  The count above it goes
+// to ctl[c_bin + 1], the bin's own count to ctl[c_bin + 2]; ctl[c_bin] = -1 when the histogram holds
+// fewer than `target` entries.  All NT threads of the group call it; every bin is read by exactly one
+// thread, which leaves it zero for the next row.
+template <int BINS, int NT, int BAR>
+__device__ __forceinline__ void find_rank_bin(uint32_t* hist, uint32_t target, int tid, uint64_t* scratch, int* ctl,
+                                              int c_bin) {
+  constexpr int PER = BINS / NT;
+  static_assert(BINS % NT == 0 && PER % 4 == 0, "bins must split into 16-byte pieces per thread");
+  // thread t owns bins BINS-1 - PER*t - j, j = 0..PER-1, i.e. words [BINS - PER (t+1), BINS - PER t)
+  uint32_t c[PER], sum = 0;
+  uint4* mine = reinterpret_cast<uint4*>(hist + BINS - PER * (tid + 1));
+#pragma unroll
+  for (int v = 0; v < PER / 4; ++v) {
+    const uint4 w = mine[v];
+    mine[v] = make_uint4(0u, 0u, 0u, 0u);
+    c[PER - 1 - 4 * v] = w.x; c[PER - 2 - 4 * v] = w.y; c[PER - 3 - 4 * v] = w.z; c[PER - 4 - 4 * v] = w.w;
+  }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) sum += c[j];
+  if (tid == 0) ctl[c_bin] = -1;
+  uint32_t total;
+  uint32_t above = group_exclusive_scan<NT, BAR, uint32_t>(sum, tid, scratch, &total);
+  if (above < target && target <= above + sum) {
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      if (above < target && target <= above + c[j]) {
+        ctl[c_bin] = BINS - 1 - PER * tid - j;
+        ctl[c_bin + 1] = (int)above;
+        ctl[c_bin + 2] = (int)c[j];
+      }
+      above += c[j];
+    }
+  }
+  group_sync<NT, BAR>();
+}
+
+// Visit the candidates of one row: finisher warp pw takes the lists of filter warps pw, pw+NP, ...;
+// four independent entries per lane are in flight at a time.
+template <int NF, int NP, typename F>
+__device__ __forceinline__ void for_each_candidate(const Candidate* lists, const int* count, int pw, int lane, F f) {
+  for (int seg = pw; seg < NF; seg += NP) {
+    const Candidate* s = lists + (size_t)seg * kWarpListCap;
+    const int n = min(count[seg], kWarpListCap);
+    for (int i0 = 0; i0 < n; i0 += 128) {
+      Candidate c[4];
+      bool v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int i = i0 + q * 32 + lane;
+        v[q] = i < n;
+        if (v[q]) c[q] = s[i];
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (v[q]) f(c[q]);
+    }
+  }
+}
+
+template <int DTYPE, int NF, int NP>
+__global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(const RowArgs a, const PipeCfg cfg) {
+  constexpr int NT_F = NF * 32, NT_P = NP * 32;
+  constexpr int BAR_F = 1, BAR_P = 2;
+  static_assert(NF <= 16 && NP * 32 * kFinItems >= kKcapMax, "group sizes");
+  using TR = PipeTraits<DTYPE>;
+  constexpr int TPS = TR::kTilesPerStage;
+  extern __shared__ unsigned char smem_raw[];
+  PipeSmem<NF> sm = carve_pipe_smem<NF>(smem_raw, cfg.n_stages, cfg.vwords);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int NS = cfg.n_stages;
+  const bool has_u = a.uncond != nullptr;
+  const float neg_inf = __int_as_float(0xff800000);
+
+  // ---- one-time set-up: barriers and the tables that must start at zero ----
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(&sm.full[s], 1);
+      mbar_init(&sm.empty[s], NF);
+    }
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(&sm.cand_full[k], NF);
+      mbar_init(&sm.cand_free[k], 1);
+    }
+    for (int k = 0; k < kCtlWords; ++k) sm.ctl[k] = 0;
+    fence_barrier_init();
+  }
+  for (int j = threadIdx.x; j < kCoarseBins; j += blockDim.x) sm.coarse[j] = 0;
+  for (int j = threadIdx.x; j < kFineBins; j += blockDim.x) sm.fine[j] = 0;
+  for (int j = threadIdx.x; j < kSelBins; j += blockDim.x) sm.sel[j] = 0;
+  for (int j = threadIdx.x; j < cfg.vwords; j += blockDim.x) sm.bitmap[j] = 0;
+  if (threadIdx.x < 32) {
+    sm.meta[0].count[threadIdx.x & 15] = 0;
+    sm.meta[1].count[threadIdx.x & 15] = 0;
+  }
+  __syncthreads();
+
+  const RowSchedule sched(a.V, cfg.sample_stride, TPS);
+  const int rows = a.B * a.W;
+  volatile int* abort_flag = sm.ctl + kCtlAbort;
+
+  if (warp == NF + NP) {
+    // ====================================== producer warp ======================================
+    int slot = 0;
+    uint32_t use = 0;   // how many times `slot` has been filled before
+    uint32_t issued = 0;
+    bool ok = true;
+    for (int row = blockIdx.x; row < rows && ok; row += gridDim.x) {
+      const int b = row / a.W, i = row - b * a.W;
+      const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
+      if (i >= L) continue;
+      const int64_t off = (int64_t)b * a.stride_b + (int64_t)i * a.stride_w;
+      const unsigned char* gc = static_cast<const unsigned char*>(a.cond) + off * TR::kElemBytes;
+      const unsigned char* gu = has_u ? static_cast<const unsigned char*>(a.uncond) + off * TR::kElemBytes : nullptr;
+      for (int s = 0; s < sched.stages; ++s) {
+        if (use > 0) ok = mbar_wait(&sm.empty[slot], (use - 1) & 1u);
+        ok = __all_sync(0xffffffffu, ok && (*abort_flag == 0));
+        if (!ok) break;
+        const int nt = sched.stage_tiles(s, TPS);
+        unsigned char* dst_c = sm.ring + (size_t)slot * TR::kStageBytes;
+        unsigned char* dst_u = dst_c + kStageArrayBytes;
+        if (lane == 0) mbar_arrive_expect_tx(&sm.full[slot], (uint32_t)nt * TR::kTileBytes * (has_u ? 2u : 1u));
+        __syncwarp();
+        if (s < sched.sample_stages) {
+          // sample tiles are isolated in the row: one copy per tile, spread over the lanes
+          for (int j = lane; j < nt; j += 32) {
+            const size_t goff = (size_t)(s * TPS + j) * sched.ss * TR::kTileBytes;
+            bulk_g2s(dst_c + (size_t)j * TR::kTileBytes, gc + goff, TR::kTileBytes, &sm.full[slot]);
+            if (has_u) bulk_g2s(dst_u + (size_t)j * TR::kTileBytes, gu + goff, TR::kTileBytes, &sm.full[slot]);
+          }
+        } else {
+          // tail tiles come in runs of SS-1 contiguous tiles: lane r copies the r-th run of the stage
+          const int t0 = TPS * (s - sched.sample_stages), t1 = t0 + nt, rl = sched.ss - 1;
+          const int run = t0 / rl + lane;
+          const int ta = max(run * rl, t0), tb = min((run + 1) * rl, t1);
+          if (ta < tb) {
+            const int g = run * sched.ss + 1 + (ta - run * rl);
+            const uint32_t bytes = (uint32_t)(tb - ta) * TR::kTileBytes;
+            const size_t goff = (size_t)g * TR::kTileBytes, soff = (size_t)(ta - t0) * TR::kTileBytes;
+            bulk_g2s(dst_c + soff, gc + goff, bytes, &sm.full[slot]);
+            if (has_u) bulk_g2s(dst_u + soff, gu + goff, bytes, &sm.full[slot]);
+          }
+        }
+        ++issued;
+        if (++slot == NS) {
+          slot = 0;
+          ++use;
+        }
+      }
+    }
+    // drain: every stage this warp armed must have landed before the CTA may exit
+    {
+      const uint32_t n_back = issued < (uint32_t)NS ? issued : (uint32_t)NS;
+      int sl = slot;
+      uint32_t us = use;
+      for (uint32_t k = 0; k < n_back; ++k) {
+        if (--sl < 0) {
+          sl = NS - 1;
+          --us;
+        }
+        mbar_wait(&sm.full[sl], us & 1u);
+      }
+      if (!ok && lane == 0) *abort_flag = 1;
+    }
+    return;
+  }
+
+  if (warp < NF) {
+    // ======================================= filter warps =======================================
+    const int tid = threadIdx.x;  // 0 .. NT_F-1
+    const int fw = warp;
+    const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
+    const bool has_t = a.inv_T != 1.0f;
+    int slot = 0;
+    uint32_t phase = 0;
+    uint32_t n_row = 0;
+    bool dead = false;
+    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+      const int b = row / a.W, i = row - b * a.W;
+      const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
+      if (i >= L || dead) continue;
+      const int buf = (int)(n_row & 1u);
+      const uint32_t buf_use = n_row >> 1;
+      RowMeta* meta = sm.meta + buf;
+      Candidate* seg = sm.lists + ((size_t)buf * NF + fw) * kWarpListCap;
+
+      // ---------------- sample stages: histogram of the order-preserving keys ----------------
+      bool ok = true;
+      {
+        int sl = slot;
+        uint32_t ph = phase;
+        for (int s = 0; s < sched.sample_stages && ok; ++s) {
+          ok = mbar_wait(&sm.full[sl], ph);
+          if (ok) {
+            const unsigned char* st_c = sm.ring + (size_t)sl * TR::kStageBytes;
+            const unsigned char* st_u = st_c + kStageArrayBytes;
+            const int nt = sched.stage_tiles(s, TPS);
+            for (int j = fw; j < nt; j += NF) {
+              float y[8];
+              tile_y8<DTYPE>(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes, has_u, has_t, lane, s2,
+                             t2, y);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) atomicAdd(&sm.coarse[float_key(canonical(y[e])) >> 21], 1u);
+            }
+          }
+          if (++sl == NS) {
+            sl = 0;
+            ph ^= 1u;
+          }
+        }
+      }
+      dead = group_any<NT_F, BAR_F>(!ok);
+      if (dead) {
+        if (tid == 0) *abort_flag = 1;
+        continue;
+      }
+      find_rank_bin<kCoarseBins, NT_F, BAR_F>(sm.coarse, (uint32_t)cfg.sample_rank, tid, sm.scan_f, sm.ctl, kCtlFBin);
+      const int cbin = sm.ctl[kCtlFBin];
+      const int fine_target = cfg.sample_rank - sm.ctl[kCtlFAbove];
+      // ---------------- second level inside the coarse bin ----------------
+      {
+        int sl = slot;
+        for (int s = 0; s < sched.sample_stages; ++s) {
+          const unsigned char* st_c = sm.ring + (size_t)sl * TR::kStageBytes;
+          const unsigned char* st_u = st_c + kStageArrayBytes;
+          const int nt = sched.stage_tiles(s, TPS);
+          for (int j = fw; j < nt; j += NF) {
+            float y[8];
+            tile_y8<DTYPE>(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes, has_u, has_t, lane, s2, t2,
+                           y);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const uint32_t k = float_key(canonical(y[e]));
+              if ((int)(k >> 21) == cbin) atomicAdd(&sm.fine[(k >> 13) & 0xffu], 1u);
+            }
+          }
+          if (++sl == NS) sl = 0;
+        }
+      }
+      group_sync<NT_F, BAR_F>();
+      if (fw == 0) {
+        // lane l owns fine bins 255-8l .. 248-8l; walk from the largest bin down
+        uint32_t c[8], sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          c[j] = sm.fine[255 - 8 * lane - j];
+          sm.fine[255 - 8 * lane - j] = 0;
+          sum += c[j];
+        }
+        uint32_t inc = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t n = __shfl_up_sync(0xffffffffu, inc, d);
+          if (lane >= d) inc += n;
+        }
+        uint32_t above = inc - sum;
+        const uint32_t target = (uint32_t)fine_target;
+        int fbin = -1;
+        if (above < target && target <= inc) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (above < target && target <= above + c[j]) fbin = 255 - 8 * lane - j;
+            above += c[j];
+          }
+        }
+        const float lowest = -3.402823466e38f;  // with this threshold every finite value is a candidate
+        const bool found = fbin >= 0 && cbin >= 0;
+        if (found) {
+          // lower edge of (coarse bin, fine bin) as a float: every value of the bin is >= it
+          const uint32_t key = ((uint32_t)cbin << 21) | ((uint32_t)fbin << 13);
+          const uint32_t bits = (key & 0x80000000u) ? (key & 0x7fffffffu) : ~key;
+          float t0 = __uint_as_float(bits);
+          if (!(t0 >= lowest)) t0 = lowest;  // edge fell on -inf or into the NaN patterns
+          sm.ctl[kCtlTau0] = __float_as_int(t0);
+        }
+        if (!__any_sync(0xffffffffu, found) && lane == 0) sm.ctl[kCtlTau0] = __float_as_int(lowest);
+      }
+      // ---------------- the candidate buffer must be back from the finisher ----------------
+      if (buf_use > 0) ok = mbar_wait(&sm.cand_free[buf], (buf_use - 1) & 1u);
+      dead = group_any<NT_F, BAR_F>(!ok);  // also publishes tau0
+      if (dead) {
+        if (tid == 0) *abort_flag = 1;
+        continue;
+      }
+      const float tau0 = __int_as_float(sm.ctl[kCtlTau0]);
+      int* wcount = &meta->count[fw];
+      if (lane == 0) *wcount = 0;
+      __syncwarp();
+      float vmax = neg_inf;
+      auto filter_tile = [&](const unsigned char* ctile, const unsigned char* utile, int id_base) {
+        float y[8];
+        tile_y8<DTYPE>(ctile, utile, has_u, has_t, lane, s2, t2, y);
+        vmax = max3(vmax, y[0], y[1]);
+        vmax = max3(vmax, y[2], y[3]);
+        vmax = max3(vmax, y[4], y[5]);
+        vmax = max3(vmax, y[6], y[7]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (y[e] >= tau0) {
+            const int pos = atomicAdd(wcount, 1);
+            if (pos < kWarpListCap) seg[pos] = Candidate{y[e], id_base + tile_elem<DTYPE>(lane, e)};
+          }
+        }
+      };
+      // ---------------- the sample tiles, now against tau0 ----------------
+      for (int s = 0; s < sched.sample_stages; ++s) {
+        const unsigned char* st_c = sm.ring + (size_t)slot * TR::kStageBytes;
+        const unsigned char* st_u = st_c + kStageArrayBytes;
+        const int nt = sched.stage_tiles(s, TPS);
+        for (int j = fw; j < nt; j += NF)
+          filter_tile(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes,
+                      sched.global_tile(s, j, TPS) * kTileElems);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[slot]);
+        if (++slot == NS) {
+          slot = 0;
+          phase ^= 1u;
+        }
+      }
+      // ---------------- the rest of the row ----------------
+      for (int s = sched.sample_stages; s < sched.stages; ++s) {
+        if (ok) ok = mbar_wait(&sm.full[slot], phase);
+        if (ok) {
+          const unsigned char* st_c = sm.ring + (size_t)slot * TR::kStageBytes;
+          const unsigned char* st_u = st_c + kStageArrayBytes;
+          const int nt = sched.stage_tiles(s, TPS);
+          for (int j = fw; j < nt; j += NF)
+            filter_tile(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes,
+                        sched.global_tile(s, j, TPS) * kTileElems);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[slot]);
+        if (++slot == NS) {
+          slot = 0;
+          phase ^= 1u;
+        }
+      }
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, d));
+      if (lane == 0) {
+        meta->vmax[fw] = vmax;
+        if (fw == 0) meta->tau0 = tau0;
+      }
+      dead = group_any<NT_F, BAR_F>(!ok);
+      if (dead) {
+        if (tid == 0) *abort_flag = 1;
+        continue;  // the buffer is not handed over: the finisher's wait runs out and marks the rows
+      }
+      if (lane == 0) mbar_arrive(&sm.cand_full[buf]);
+      ++n_row;
+    }
+    return;
+  }
+
+  // ======================================= finisher warps =======================================
+  const int tid = threadIdx.x - NT_F;  // 0 .. NT_P-1
+  const int pw = tid >> 5;
+  uint32_t n_row = 0;
+  bool dead = false;
+  for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    const int b = row / a.W, i = row - b * a.W;
+    const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
+    RowScratch* rs = a.scratch + row;
+    if (i >= L) {
+      if (tid == 0) {
+        a.out_cnt[row] = 0;
+        *rs = RowScratch{0.0f, -1, 0.0f, 0};
+      }
+      continue;
+    }
+    const int kcap = a.kcap;
+    const int buf = (int)(n_row & 1u);
+    const int draft = a.drafts ? a.drafts[row] : -1;
+    if (!dead) dead = !mbar_wait(&sm.cand_full[buf], (n_row >> 1) & 1u);
+    dead = group_any<NT_P, BAR_P>(dead || (*abort_flag != 0));
+    if (dead) {
+      if (tid == 0) {
+        *abort_flag = 1;
+        a.out_cnt[row] = 0;
+        *rs = RowScratch{0.0f, -1, 0.0f, kRowStatusTimeout};
+      }
+      continue;
+    }
+    const RowMeta* meta = sm.meta + buf;
+    const Candidate* lists = sm.lists + (size_t)buf * NF * kWarpListCap;
+    const float tau0 = meta->tau0;
+    int n_total = 0;
+    bool fallback = kcap > kKcapMax;
+    float vmax = neg_inf;
+#pragma unroll
+    for (int w = 0; w < NF; ++w) {
+      const int c = meta->count[w];
+      fallback |= c > kWarpListCap;
+      n_total += c;
+      vmax = fmaxf(vmax, meta->vmax[w]);
+    }
+    fallback |= n_total < kcap;
+    fallback |= !(vmax <= 3.402823466e38f);  // an infinite logit: the any-shape path decides what the row is
+
+    int tbin = 0, need = 0, nbin = 0;
+    const float range = __fsub_rn(vmax, tau0);
+    const float scale = range > 0.0f ? __fdiv_rn((float)kSelBins * 0.999f, range) : 0.0f;
+    // linear bins over [tau0, vmax]; monotone in y, so a higher bin holds strictly larger values
+    auto bin_of = [&](float y) {
+      const int q = __float2int_rd(__fmul_rn(__fsub_rn(y, tau0), scale));
+      return min(max(q, 0), kSelBins - 1);
+    };
+    if (!fallback) {
+      for_each_candidate<NF, NP>(lists, meta->count, pw, lane,
+                                 [&](const Candidate& c) { atomicAdd(&sm.sel[bin_of(c.y)], 1u); });
+      group_sync<NT_P, BAR_P>();
+      find_rank_bin<kSelBins, NT_P, BAR_P>(sm.sel, (uint32_t)kcap, tid, sm.scan_p, sm.ctl, kCtlPBin);
+      tbin = sm.ctl[kCtlPBin];
+      need = kcap - sm.ctl[kCtlPAbove];  // members of the threshold bin that survive
+      nbin = sm.ctl[kCtlPCount];
+      if (tbin < 0 || nbin > kBinListCap) fallback = true;
+    }
+    uint32_t wsum = 0, wrun = 0;
+    const int wper = (cfg.vwords + NT_P - 1) / NT_P;
+    const int w0 = min(tid * wper, cfg.vwords), w1 = min(w0 + wper, cfg.vwords);
+    if (!fallback) {
+      // ---- survivors into the bitmap over token ids: everything above the threshold bin, and the
+      //      `need` best of the bin itself by (y descending, id ascending) ----
+      for_each_candidate<NF, NP>(lists, meta->count, pw, lane, [&](const Candidate& c) {
+        const int q = bin_of(c.y);
+        if (q > tbin) atomicOr(&sm.bitmap[c.id >> 5], 1u << (c.id & 31));
+        else if (q == tbin) sm.binlist[atomicAdd(&sm.ctl[kCtlGather], 1)] = Candidate{canonical(c.y), c.id};
+      });
+      group_sync<NT_P, BAR_P>();
+      for (int x = tid; x < nbin; x += NT_P) {
+        const Candidate me = sm.binlist[x];
+        int rank = 0;
+        for (int z = 0; z < nbin; ++z) {
+          const Candidate o = sm.binlist[z];
+          rank += (o.y > me.y || (o.y == me.y && o.id < me.id)) ? 1 : 0;
+        }
+        if (rank < need) atomicOr(&sm.bitmap[me.id >> 5], 1u << (me.id & 31));
+      }
+      group_sync<NT_P, BAR_P>();
+      // ---- exclusive prefix of the per-word popcounts; each thread owns a contiguous run of words ----
+      for (int w = w0; w < w1; ++w) wsum += __popc(sm.bitmap[w]);
+      uint32_t total;
+      wrun = group_exclusive_scan<NT_P, BAR_P, uint32_t>(wsum, tid, sm.scan_p, &total);
+      for (int w = w0; w < w1; ++w) {
+        sm.wprefix[w] = (uint16_t)wrun;
+        wrun += __popc(sm.bitmap[w]);
+      }
+      if (total != (uint32_t)kcap) fallback = true;  // cannot happen; keep the result exact anyway
+      group_sync<NT_P, BAR_P>();
+    }
+    if (!fallback) {
+      // ---- softmax numerators into ascending-id order ----
+      for_each_candidate<NF, NP>(lists, meta->count, pw, lane, [&](const Candidate& c) {
+        const uint32_t w = sm.bitmap[c.id >> 5];
+        const uint32_t bit = 1u << (c.id & 31);
+        if (w & bit) {
+          const int pos = (int)sm.wprefix[c.id >> 5] + __popc(w & (bit - 1u));
+          sm.st_ids[pos] = c.id;
+          sm.st_vals[pos] = exp_diff(canonical(c.y), vmax);
+        }
+      });
+    }
+    group_sync<NT_P, BAR_P>();
+    // the candidate lists are not read again: hand the buffer back, leave the tables clean
+    if (tid == 0) {
+      mbar_arrive(&sm.cand_free[buf]);
+      sm.ctl[kCtlGather] = 0;
+      sm.ctl[kCtlPtok] = 0;
+      sm.ctl[kCtlFoundId] = -1;
+    }
+    ++n_row;
+    for (int w = w0; w < w1; ++w) sm.bitmap[w] = 0;
+    if (fallback) {
+      // exact any-shape path from global memory (the row is still in L2)
+      group_sync<NT_P, BAR_P>();
+      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_ids));
+      continue;
+    }
+    // ---- normalise, write the row, draw from it ----
+    const int k0 = tid * kFinItems;
+    float e[kFinItems];
+    int ids[kFinItems];
+    float zpart = 0.0f;
+#pragma unroll
+    for (int j = 0; j < kFinItems; ++j) {
+      const bool in = k0 + j < kcap;
+      e[j] = in ? sm.st_vals[k0 + j] : 0.0f;
+      ids[j] = in ? sm.st_ids[k0 + j] : -1;
+      zpart += e[j];
+    }
+    const float Z = group_sum_f32<NT_P, BAR_P>(zpart, tid, sm.scan_p);
+    int32_t* out_ids = a.out_ids + (size_t)row * kcap;
+    float* out_vals = a.out_vals + (size_t)row * kcap;
+    uint64_t wgt[kFinItems], wloc = 0;
+    float p[kFinItems];
+#pragma unroll
+    for (int j = 0; j < kFinItems; ++j) {
+      p[j] = __fdiv_rn(e[j], Z);
+      wgt[j] = fixed_weight(p[j]);
+      wloc += wgt[j];
+      if (ids[j] == draft && ids[j] >= 0) sm.ctl[kCtlPtok] = __float_as_int(p[j]);
+    }
+    if ((kcap & 3) == 0 && k0 + kFinItems <= kcap) {
+      int4* oi = reinterpret_cast<int4*>(out_ids + k0);
+      float4* ov = reinterpret_cast<float4*>(out_vals + k0);
+      oi[0] = make_int4(ids[0], ids[1], ids[2], ids[3]);
+      oi[1] = make_int4(ids[4], ids[5], ids[6], ids[7]);
+      ov[0] = make_float4(p[0], p[1], p[2], p[3]);
+      ov[1] = make_float4(p[4], p[5], p[6], p[7]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < kFinItems; ++j) {
+        if (k0 + j < kcap) {
+          out_ids[k0 + j] = ids[j];
+          out_vals[k0 + j] = p[j];
+        }
+      }
+    }
+    // the row's own draw from p_i: fixed-point inverse CDF in ascending-id order
+    const int pos = (a.pos_base ? a.pos_base[b] : 0) + i;
+    const int iter = a.iteration ? a.iteration[b] : a.iteration0;
+    const Philox4 rnd = philox4x32_10((uint32_t)pos, (uint32_t)(a.seq_base + b), (uint32_t)iter, (uint32_t)a.purpose,
+                                      a.seed_lo, a.seed_hi);
+    uint64_t T;
+    const uint64_t lo = group_exclusive_scan<NT_P, BAR_P, uint64_t>(wloc, tid, sm.scan_p, &T);
+    const uint64_t t = __umul64hi(random64(rnd), T);
+    if (T > 0 && t >= lo && t < lo + wloc) {
+      uint64_t run = lo;
+      int j = 0;
+#pragma unroll
+      for (int q = 0; q < kFinItems; ++q) {
+        run += wgt[q];
+        if (t >= run) j = q + 1;
+      }
+      // j < kFinItems because t < lo + wloc
+      int fid = ids[0];
+      float fp = p[0];
+#pragma unroll
+      for (int q = 1; q < kFinItems; ++q) {
+        if (q == j) {
+          fid = ids[q];
+          fp = p[q];
+        }
+      }
+      sm.ctl[kCtlFoundId] = fid;
+      sm.ctl[kCtlFoundP] = __float_as_int(fp);
+    }
+    if (T == 0 && tid == 0) {  // all weights rounded to zero: take the first entry
+      sm.ctl[kCtlFoundId] = ids[0];
+      sm.ctl[kCtlFoundP] = __float_as_int(p[0]);
+    }
+    group_sync<NT_P, BAR_P>();
+    if (tid == 0) {
+      a.out_cnt[row] = kcap;
+      *rs = RowScratch{__int_as_float(sm.ctl[kCtlPtok]), sm.ctl[kCtlFoundId], __int_as_float(sm.ctl[kCtlFoundP]), 0};
+    }
+    group_sync<NT_P, BAR_P>();
+  }
+}
+
+}  // namespace sjd

@@ -10,7 +10,7 @@
 
 #include "device_utils.cuh"
 #include "row_kernels.cuh"
-#include "rows_stream.cuh"
+#include "rows_pipeline.cuh"
 #include "verify_kernel.cuh"
 
 #include <cmath>
@@ -41,54 +41,60 @@ int sm_count() {
   return cached;
 }
 
-constexpr int kStreamConsumerWarps = 16;
-constexpr int kStreamStages = 3;
+constexpr int kFilterWarps = 8;
+constexpr int kFinisherWarps = 8;
+constexpr int kMaxStages = 12;
+constexpr size_t kSmemLimit = 227u * 1024u;
 
-// Decide whether the single-pass streaming kernel can take this shape, and with which sampling
+// Decide whether the single-pass pipelined kernel can take this shape, and with which sampling
 // parameters.  The sample is every SS-th 256-element tile of a row; its rank-m value (from the top)
-// becomes the candidate threshold.  m is chosen six standard deviations above K/SS, so that a row with
-// exchangeable entries fails to deliver K candidates with probability below 1e-9 (such a row is redone
-// by the generic path, never answered wrongly).
-bool plan_stream(const sjd_params* P, int kcap, sjd::StreamCfg* cfg, size_t* smem) {
+// becomes the candidate threshold.  m is chosen 4.5 standard deviations above K/SS, so that a row with
+// exchangeable entries fails to deliver K candidates with probability below 1e-5 (such a row is redone
+// by the any-shape path, never answered wrongly), and the candidate lists must hold the expected count
+// six standard deviations above its mean.
+bool plan_pipeline(const sjd_params* P, int kcap, sjd::PipeCfg* cfg, size_t* smem) {
   const int V = P->V;
-  const int tps = P->logits_dtype == SJD_BF16 ? 32 : 16;
-  if (kcap > sjd::kStageKcapMax || V % sjd::kTileElems != 0) return false;
+  if (kcap > sjd::kKcapMax || V % sjd::kTileElems != 0) return false;
+  const int tile_bytes = sjd::kTileElems * (P->logits_dtype == SJD_BF16 ? 2 : 4);
+  const int tps = sjd::kStageArrayBytes / tile_bytes;
   const int tiles = V / sjd::kTileElems;
-  int ss = 0;
-  for (int cand : {8, 16, 32}) {
-    if (tiles % cand == 0 && tiles / cand <= tps) {
-      ss = cand;
-      break;
-    }
+  const int vwords = V / 32;
+  const size_t fixed = sjd::pipe_smem_fixed_bytes(kFilterWarps, vwords);
+  if (fixed + 4 * 2 * (size_t)sjd::kStageArrayBytes > kSmemLimit) return false;
+  int ns = (int)((kSmemLimit - fixed) / (2 * (size_t)sjd::kStageArrayBytes));
+  if (ns > kMaxStages) ns = kMaxStages;
+  for (int ss : {8, 16, 32}) {
+    if (tiles % ss != 0) continue;
+    const int sample_tiles = tiles / ss;
+    const int sample_stages = (sample_tiles + tps - 1) / tps;
+    if (sample_stages + 3 > ns) continue;
+    const int n_sample = V / ss;
+    const double a = (double)kcap / ss;
+    const double root = 2.25 + std::sqrt(2.25 * 2.25 + a);
+    const int m = (int)std::ceil(root * root);
+    if (m > n_sample / 2) continue;
+    const double expect = ((double)m + 6.0 * std::sqrt((double)m)) * ss;
+    if (expect > 0.9 * (double)sjd::kWarpListCap * kFilterWarps) continue;
+    cfg->sample_stride = ss;
+    cfg->sample_rank = m;
+    cfg->n_stages = ns;
+    cfg->vwords = vwords;
+    *smem = sjd::pipe_smem_bytes(ns, kFilterWarps, vwords);
+    return true;
   }
-  if (ss == 0) return false;
-  const int n_sample = V / ss;
-  const double a = (double)kcap / ss;
-  const double root = 3.0 + std::sqrt(9.0 + a);
-  const int m = (int)std::ceil(root * root);
-  if (m > n_sample / 2) return false;
-  // expected candidates, six sigma above, must fit the per-thread lists with room to spare
-  const double expect = ((double)m + 6.0 * std::sqrt((double)m)) * ss * 1.25;
-  const int nt = kStreamConsumerWarps * 32;
-  if (expect > 0.75 * (double)sjd::kLaneListCap * nt) return false;
-  cfg->sample_stride = ss;
-  cfg->sample_rank = m;
-  cfg->n_stages = kStreamStages;
-  cfg->vwords = V / 32;
-  *smem = sjd::stream_smem_bytes(cfg->n_stages, nt, cfg->vwords);
-  return *smem <= 227u * 1024u;
+  return false;
 }
 
 template <int DTYPE>
-cudaError_t launch_stream(const sjd::RowArgs& ra, const sjd::StreamCfg& cfg, size_t smem, int grid, cudaStream_t st) {
-  auto kern = sjd::rows_stream_kernel<DTYPE, kStreamConsumerWarps>;
+cudaError_t launch_pipeline(const sjd::RowArgs& ra, const sjd::PipeCfg& cfg, size_t smem, int grid, cudaStream_t st) {
+  auto kern = sjd::rows_pipeline_kernel<DTYPE, kFilterWarps, kFinisherWarps>;
   static bool configured = false;  // per instantiation; the attribute is sticky for the process
   if (!configured) {
-    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<grid, kStreamConsumerWarps * 32 + 32, smem, st>>>(ra, cfg);
+  kern<<<grid, (kFilterWarps + kFinisherWarps + 1) * 32, smem, st>>>(ra, cfg);
   return cudaGetLastError();
 }
 
@@ -182,13 +188,13 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
     if (e != cudaSuccess) return cuda_fail(e, "event record");
   }
   {
-    sjd::StreamCfg cfg;
+    sjd::PipeCfg cfg;
     size_t smem = 0;
     cudaError_t e;
-    if (!(P->flags & SJD_FLAG_FORCE_GENERIC) && plan_stream(P, kcap, &cfg, &smem)) {
+    if (!(P->flags & SJD_FLAG_FORCE_GENERIC) && plan_pipeline(P, kcap, &cfg, &smem)) {
       const int grid = rows < sm_count() ? rows : sm_count();
-      e = P->logits_dtype == SJD_BF16 ? launch_stream<1>(ra, cfg, smem, grid, stream)
-                                      : launch_stream<0>(ra, cfg, smem, grid, stream);
+      e = P->logits_dtype == SJD_BF16 ? launch_pipeline<1>(ra, cfg, smem, grid, stream)
+                                      : launch_pipeline<0>(ra, cfg, smem, grid, stream);
     } else {
       const int grid = rows < 4 * sm_count() ? rows : 4 * sm_count();
       if (P->logits_dtype == SJD_BF16)
