@@ -44,6 +44,7 @@ extern "C" {
 
 #define SJD_VERSION 1
 #define SJD_W_MAX 512 /* largest window of the paper's window-size ablation */
+#define SJD_STATIC_MAX_ROWS 16384 /* largest B*W sjd_step_static() accepts */
 
 /* logits_dtype */
 #define SJD_F32 0
@@ -158,6 +159,32 @@ size_t sjd_workspace_bytes(const sjd_params* params);
 int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* drafts,
              const sjd_probs* draft_probs, const sjd_params* params, uint64_t philox_seed,
              int32_t* out_accept_len, int32_t* out_tokens, sjd_probs* out_probs);
+
+/*
+ * sjd_step() for callers that cannot hand over a workspace.  (The paper has no counterpart: this is a
+ * convenience of this library, not a step of the method.)
+ *
+ * Some hosts of this library may not allocate device memory at the point where they call it: a plugin
+ * that runs inside another framework's stream callback or inside a memory pool it does not own, a
+ * serving loop that has frozen its allocator after start-up, a process whose device memory is handed out
+ * by a supervisor.  For them the scratch of the step (one 16-byte record per window row) lives in a
+ * fixed array inside the library's device image, SJD_STATIC_MAX_ROWS records long (256 KiB; every GPU that
+ * loads the library holds it until the process exits).  Arguments, results and error codes are those of
+ * sjd_step(), except that params->workspace and params->workspace_bytes are ignored and that
+ * B * W > SJD_STATIC_MAX_ROWS is refused with SJD_ERR_CAPACITY, nothing enqueued.  The call itself never
+ * calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current) and remembers it; make that first call outside any stream capture.
+ *
+ * All calls on a device share the one array.  Nothing in it has to start at zero (the row stage writes
+ * every record before the verification stage reads it), and it keeps the last call's contents.  Two calls
+ * whose kernels can overlap on the GPU (different streams without an ordering between them) race on it:
+ * order them, or use sjd_step() with separate workspaces.
+ */
+int sjd_step_static(const void* logits_cond, const void* logits_uncond, const int32_t* drafts,
+                    const sjd_probs* draft_probs, const sjd_params* params, uint64_t philox_seed,
+                    int32_t* out_accept_len, int32_t* out_tokens, sjd_probs* out_probs);
 
 /*
  * Host-buffer variant for callers whose logits and window state live in host memory.

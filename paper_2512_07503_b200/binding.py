@@ -60,6 +60,8 @@ def lib() -> C.CDLL:
         L.sjd_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs), C.POINTER(sjd_params),
                                C.c_uint64, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs)]
         L.sjd_step.restype = C.c_int
+        L.sjd_step_static.argtypes = L.sjd_step.argtypes
+        L.sjd_step_static.restype = C.c_int
         _lib = L
     return _lib
 
@@ -184,6 +186,29 @@ def sjd_step(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor], d
                               _opt_ptr(drafts), C.byref(q) if q is not None else None, C.byref(params),
                               int(philox_seed) & 0xFFFFFFFFFFFFFFFF, _opt_ptr(out_accept_len), _opt_ptr(out_tokens),
                               C.byref(o))
+    _check(code)
+
+
+SJD_STATIC_MAX_ROWS = 16384
+
+
+def sjd_step_static(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor], drafts: Optional[torch.Tensor],
+                    draft_probs: Optional[DeviceProbs], params: sjd_params, philox_seed: int,
+                    out_accept_len: torch.Tensor, out_tokens: torch.Tensor, out_probs: DeviceProbs) -> None:
+    """``sjd_step`` without a caller-supplied workspace, for hosts that may not allocate device memory where
+    they call the library (a frozen allocator, a pool they do not own).  The scratch is a fixed array inside
+    the library, good for B*W <= SJD_STATIC_MAX_ROWS; larger problems raise.  ``params.workspace`` is ignored.
+    Calls on one device share that array: do not let two of them overlap on the GPU."""
+    if not logits_cond.is_cuda:
+        raise SjdError("logits must live on a CUDA device")
+    q = draft_probs.c_struct() if draft_probs is not None else None
+    o = out_probs.c_struct()
+    with torch.cuda.device(logits_cond.device):
+        code = lib().sjd_step_static(logits_cond.data_ptr(),
+                                     None if logits_uncond is None else logits_uncond.data_ptr(), _opt_ptr(drafts),
+                                     C.byref(q) if q is not None else None, C.byref(params),
+                                     int(philox_seed) & 0xFFFFFFFFFFFFFFFF, _opt_ptr(out_accept_len),
+                                     _opt_ptr(out_tokens), C.byref(o))
     _check(code)
 
 

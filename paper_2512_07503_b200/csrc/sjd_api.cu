@@ -7,6 +7,7 @@
 #include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "device_utils.cuh"
 #include "row_kernels.cuh"
@@ -96,6 +97,34 @@ cudaError_t launch_pipeline(const sjd::RowArgs& ra, const sjd::PipeCfg& cfg, siz
   }
   kern<<<grid, (kFilterWarps + kFinisherWarps + 1) * 32, smem, st>>>(ra, cfg);
   return cudaGetLastError();
+}
+
+// Scratch of sjd_step_static(): lives in the library's device image, so every GPU that loads the library
+// holds these bytes until the process exits.  Sized for SJD_STATIC_MAX_ROWS rows of RowScratch.
+constexpr size_t kStaticScratchBytes = (((size_t)SJD_STATIC_MAX_ROWS * sizeof(sjd::RowScratch) + 256) + 255) & ~(size_t)255;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_scratch_addr[kMaxDevices] = {};  // device address of g_static_scratch, per device ordinal
+
+// Device address of the static scratch on the CURRENT device.  In host code the symbol's name is only a
+// handle; the address a kernel can use comes from cudaGetSymbolAddress(), asked once per device.
+int static_scratch_address(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  if (dev < 0 || dev >= kMaxDevices) return SJD_ERR_CAPACITY;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static scratch)");
+    if (p == nullptr || (reinterpret_cast<uintptr_t>(p) & 255u) != 0) return SJD_ERR_WORKSPACE;
+    g_static_scratch_addr[dev] = p;
+  }
+  *out = g_static_scratch_addr[dev];
+  return SJD_OK;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -242,6 +271,22 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
     ++g_launches;
   }
   return SJD_OK;
+}
+
+int sjd_step_static(const void* logits_cond, const void* logits_uncond, const int32_t* drafts,
+                    const sjd_probs* draft_probs, const sjd_params* P, uint64_t philox_seed, int32_t* out_accept_len,
+                    int32_t* out_tokens, sjd_probs* out_probs) {
+  if (!P) return SJD_ERR_NULL;
+  if (P->struct_size != (int32_t)sizeof(sjd_params)) return SJD_ERR_STRUCT;
+  if (P->B < 0 || P->W < 1 || P->W > SJD_W_MAX) return SJD_ERR_SHAPE;
+  if ((int64_t)P->B * (int64_t)P->W > (int64_t)SJD_STATIC_MAX_ROWS) return SJD_ERR_CAPACITY;
+  void* scratch = nullptr;
+  const int rc = static_scratch_address(&scratch);
+  if (rc != SJD_OK) return rc;
+  sjd_params Q = *P;
+  Q.workspace = scratch;
+  Q.workspace_bytes = kStaticScratchBytes;
+  return sjd_step(logits_cond, logits_uncond, drafts, draft_probs, &Q, philox_seed, out_accept_len, out_tokens, out_probs);
 }
 
 }  // extern "C"
