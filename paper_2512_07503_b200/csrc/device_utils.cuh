@@ -278,4 +278,71 @@ __device__ __forceinline__ int group_icdf(WeightFn weight, int n, uint64_t R, in
   return k;
 }
 
+// ------------------------------------------------------------------------------------------------
+// One-barrier variants.  `scratch` holds two banks of 32 uint64 that successive calls alternate
+// between (`flip`, kept by the caller, starts at 0 and must be passed to every call of the group in the
+// same order by all its threads): a thread can be at most one barrier ahead of the slowest one, so
+// the bank it writes is never the one a slower thread still reads.
+// ------------------------------------------------------------------------------------------------
+template <int NT, int BAR, typename T>
+__device__ __forceinline__ T group_scan1(T v, int tid, uint64_t* scratch, int& flip, T* total) {
+  constexpr int NW = NT / 32;
+  const int lane = tid & 31, warp = tid >> 5;
+  T inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    T n;
+    if (sizeof(T) == 8) n = (T)shfl_up_u64((uint64_t)inc, d);
+    else n = (T)__shfl_up_sync(0xffffffffu, (uint32_t)inc, d);
+    if (lane >= d) inc += n;
+  }
+  uint64_t* bank = scratch + (flip ? 32 : 0);
+  flip ^= 1;
+  if (lane == 31) bank[warp] = (uint64_t)inc;
+  group_sync<NT, BAR>();
+  T base = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) {
+    const T x = (T)bank[w];
+    tot += x;
+    if (w < warp) base += x;
+  }
+  *total = tot;
+  return base + inc - v;
+}
+
+// Sum in a fixed order (lanes by butterfly, warps in index order): the same value in every thread and in
+// every run.
+template <int NT, int BAR>
+__device__ __forceinline__ float group_sum1_f32(float v, int tid, uint64_t* scratch, int& flip) {
+  constexpr int NW = NT / 32;
+  const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+  float* bank = reinterpret_cast<float*>(scratch + (flip ? 32 : 0));
+  flip ^= 1;
+  if (lane == 0) bank[warp] = v;
+  group_sync<NT, BAR>();
+  float t = 0.0f;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) t += bank[w];
+  return t;
+}
+
+template <int NT, int BAR>
+__device__ __forceinline__ float group_max1_f32(float v, int tid, uint64_t* scratch, int& flip) {
+  constexpr int NW = NT / 32;
+  const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, d));
+  float* bank = reinterpret_cast<float*>(scratch + (flip ? 32 : 0));
+  flip ^= 1;
+  if (lane == 0) bank[warp] = v;
+  group_sync<NT, BAR>();
+  float t = __int_as_float(0xff800000);
+#pragma unroll
+  for (int w = 0; w < NW; ++w) t = fmaxf(t, bank[w]);
+  return t;
+}
+
 }  // namespace sjd

@@ -7,17 +7,20 @@
 //                       copies (cp.async.bulk, completion on mbarriers; no multicast, own CTA only).
 //   filter (NF warps)   turns the staged bf16/fp32 pairs into merged logits y and keeps only the few per
 //                       cent that can still be in the top-K.  The first stages of a row are a strided
-//                       SAMPLE of it (every SS-th 256-element tile); a two-level histogram of the
-//                       sample's order-preserving keys gives the threshold tau0 whose rank in the sample
-//                       is high enough that at least K elements of the row reach it (a row for which
-//                       that fails is redone exactly, see below).  Every element with y >= tau0 is
-//                       appended to the warp's candidate list in shared memory.
-//   finisher (NP warps) works on the PREVIOUS row's candidates while the filter streams the next row:
-//                       exact K-th largest (linear-bin histogram + ranking inside the threshold bin,
-//                       ties to the lower id), ascending-id order through a bitmap over token ids,
-//                       softmax, coalesced output, and the row's own inverse-CDF draw.
+//                       SAMPLE of it (every SS-th 256-element tile).  The maxima of the sample's groups
+//                       of eight give a floor f below the sample's rank-m value; a linear histogram of
+//                       the sample elements above f then gives the threshold tau0 whose rank in the sample
+//                       is m, high enough that at least K elements of the row reach it (a row for which
+//                       that fails is redone exactly, see below).  Pairs of neighbouring elements whose
+//                       larger one reaches tau0 are appended to a per-thread list with branch-free
+//                       arithmetic: the pair is always stored at the thread's cursor and the cursor
+//                       advances only for a hit; one bit per pair records where the hits were.
+//   finisher (NP warps) works on the PREVIOUS row while the filter streams the next one: turns lists
+//                       and hit bits into a dense candidate list, finds the exact K-th largest
+//                       (linear-bin histogram + ranking inside the threshold bin, ties to the lower
+//                       id), orders the survivors by token id through a bitmap, and does softmax,
+//                       coalesced output and the row's own inverse-CDF draw.
 //
-// Candidate lists are double buffered; filter and finisher hand them over through two mbarrier pairs.
 // A row whose candidates do not contain the top-K for sure (fewer than K of them) or do not fit the
 // on-chip capacities is redone by row_generic() from global memory: the result is exact for any input.
 //
@@ -32,10 +35,13 @@ namespace sjd {
 
 constexpr int kTileElems = 256;           // elements per tile: one warp iteration, 8 per lane
 constexpr int kStageArrayBytes = 8192;    // bytes of ONE logits array in a ring stage
-constexpr int kCoarseBins = 2048;         // sample histogram, level 1: key >> 21
-constexpr int kFineBins = 256;            // sample histogram, level 2: (key >> 13) & 0xff inside one coarse bin
+constexpr int kHistBins = 2048;           // filter's sample histogram (group maxima by key, then linear bins)
 constexpr int kSelBins = 2048;            // finisher's linear bins over [tau0, max]
-constexpr int kWarpListCap = 512;         // candidates one filter warp can hold for a row
+constexpr int kListCap = 32;              // pair entries per filter thread and row (the last four are slack
+                                          // for the unconditional stores of one tile)
+constexpr int kMaskWordsMax = 8;          // 32 hit bits each: up to 64 tiles per filter warp and row
+constexpr int kItersMax = 64;
+constexpr int kDenseCap = 3072;           // candidates the finisher can hold for a row
 constexpr int kBinListCap = 512;          // members of the threshold bin ranked by brute force
 constexpr int kKcapMax = 2048;            // largest kcap the on-chip path stages
 constexpr int kFinItems = 8;              // staged entries per finisher thread (kKcapMax / finisher threads)
@@ -47,6 +53,7 @@ struct PipeCfg {
   int sample_rank;    // m: rank (from the top) within the sample that fixes tau0
   int n_stages;       // ring depth
   int vwords;         // V / 32
+  int mask_words;     // 32-bit words of hit bits per filter thread and row
 };
 
 struct Candidate {
@@ -211,93 +218,94 @@ __device__ __forceinline__ void tile_y8(const unsigned char* ctile, const unsign
 // Shared-memory layout (dynamic)
 // ---------------------------------------------------------------------------------------------------
 enum {
-  kCtlAbort = 0,      // a bounded wait gave up somewhere in this CTA
-  kCtlFBin, kCtlFAbove, kCtlFCount, kCtlTau0,          // filter group
-  kCtlPBin, kCtlPAbove, kCtlPCount, kCtlGather,        // finisher group
-  kCtlPtok, kCtlFoundId, kCtlFoundP,
+  kCtlAbort = 0,  // a bounded wait gave up somewhere in this CTA
+  // filter group
+  kCtlFBin, kCtlFAbove, kCtlFCount, kCtlTau0, kCtlSmaxKey,
+  // handed from the filter to the finisher with the row
+  kCtlRowTau0, kCtlRowOverflow,
+  // finisher group
+  kCtlPBin, kCtlPAbove, kCtlPCount, kCtlGather, kCtlPtok, kCtlFoundId, kCtlFoundP,
   kCtlWords = 16
-};
-
-struct RowMeta {      // what the filter tells the finisher about a row, one per candidate buffer
-  float tau0;
-  float vmax[16];     // per filter warp: largest y of the tiles it saw
-  int count[16];      // per filter warp: candidates appended (may exceed kWarpListCap: overflow)
 };
 
 template <int NF>
 struct PipeSmem {
   uint64_t* full;       // [n_stages]  ring: data landed
   uint64_t* empty;      // [n_stages]  ring: all filter warps done with the stage
-  uint64_t* cand_full;  // [2]         candidate buffer handed to the finisher
-  uint64_t* cand_free;  // [2]         candidate buffer handed back
+  uint64_t* cand_full;  // lists and hit bits handed to the finisher
+  uint64_t* cand_free;  // ... and handed back
   unsigned char* ring;  // [n_stages][2][kStageArrayBytes]
-  Candidate* lists;     // [2][NF][kWarpListCap]
-  RowMeta* meta;        // [2]
-  uint32_t* coarse;     // [kCoarseBins]   (filter)
-  uint32_t* fine;       // [kFineBins]     (filter)
-  uint32_t* sel;        // [kSelBins]      (finisher)
+  uint64_t* ylist;      // [kListCap][NF*32]        pair entries, one column per filter thread
+  uint32_t* masks;      // [mask_words][NF*32]      inverted hit bits, first pair in the top bit
+  uint16_t* tile_of;    // [NF][kItersMax]          global tile of a filter warp's it-th tile of a row
+  uint32_t* hist;       // [kHistBins]     (filter)
+  Candidate* dense;     // [kDenseCap]     (finisher)
+  int32_t* st_ids;      // [kKcapMax]      (finisher) staging, ascending id
+  float* st_vals;       // [kKcapMax]
+  uint32_t* sel;        // [kSelBins]      (finisher) = st_ids: dead before the staging is written
+  Candidate* binlist;   // [kBinListCap]   (finisher) = st_vals: likewise
   uint32_t* bitmap;     // [vwords]        (finisher)
   uint16_t* wprefix;    // [vwords]        (finisher)
-  Candidate* binlist;   // [kBinListCap]   (finisher)
-  int32_t* st_ids;      // [kKcapMax]      (finisher)
-  float* st_vals;       // [kKcapMax]      (finisher)
   uint64_t* scan_f;     // group scratch, filter
   uint64_t* scan_p;     // group scratch, finisher
   int* ctl;             // control words
 };
 
-__host__ __device__ inline size_t pipe_smem_fixed_bytes(int NF, int vwords) {
+__host__ __device__ inline size_t pipe_smem_fixed_bytes(int NF, int vwords, int mask_words) {
   size_t b = 0;
-  b += 32 * 8;                                          // mbarriers (2 per ring stage + 4)
-  b += (size_t)2 * NF * kWarpListCap * sizeof(Candidate);
-  b += 2 * sizeof(RowMeta);
-  b += (size_t)(kCoarseBins + kFineBins + kSelBins) * 4;
-  b += (size_t)vwords * 4 + (size_t)vwords * 2;
-  b += (size_t)kBinListCap * sizeof(Candidate);
+  b += 32 * 8;                                           // mbarriers (2 per ring stage + 2)
+  b += (size_t)kListCap * NF * 32 * 8;                   // ylist
+  b += (size_t)mask_words * NF * 32 * 4;                 // masks
+  b += (size_t)NF * kItersMax * 2;                       // tile_of
+  b += (size_t)kHistBins * 4;
+  b += (size_t)kDenseCap * sizeof(Candidate);
   b += (size_t)kKcapMax * 8;
+  b += (size_t)vwords * 4 + (size_t)vwords * 2;
   b += 2 * (2 * 32 + 8) * 8;
   b += kCtlWords * 4;
   return b + 128;  // alignment slack
 }
-__host__ __device__ inline size_t pipe_smem_bytes(int n_stages, int NF, int vwords) {
-  return pipe_smem_fixed_bytes(NF, vwords) + (size_t)n_stages * 2 * kStageArrayBytes;
+__host__ __device__ inline size_t pipe_smem_bytes(int n_stages, int NF, int vwords, int mask_words) {
+  return pipe_smem_fixed_bytes(NF, vwords, mask_words) + (size_t)n_stages * 2 * kStageArrayBytes;
 }
 
 template <int NF>
-__device__ __forceinline__ PipeSmem<NF> carve_pipe_smem(unsigned char* base, int n_stages, int vwords) {
+__device__ __forceinline__ PipeSmem<NF> carve_pipe_smem(unsigned char* base, int n_stages, int vwords, int mask_words) {
+  static_assert(sizeof(uint32_t) * kSelBins <= sizeof(int32_t) * kKcapMax, "sel must fit under st_ids");
+  static_assert(sizeof(Candidate) * kBinListCap <= sizeof(float) * kKcapMax, "binlist must fit under st_vals");
   PipeSmem<NF> s;
   uintptr_t p = (reinterpret_cast<uintptr_t>(base) + 127) & ~(uintptr_t)127;
   s.ring = reinterpret_cast<unsigned char*>(p);
   p += (size_t)n_stages * 2 * kStageArrayBytes;
-  s.lists = reinterpret_cast<Candidate*>(p);
-  p += (size_t)2 * NF * kWarpListCap * sizeof(Candidate);
+  s.ylist = reinterpret_cast<uint64_t*>(p);
+  p += (size_t)kListCap * NF * 32 * 8;
+  s.dense = reinterpret_cast<Candidate*>(p);
+  p += (size_t)kDenseCap * sizeof(Candidate);
   s.st_ids = reinterpret_cast<int32_t*>(p);
+  s.sel = reinterpret_cast<uint32_t*>(p);
   p += (size_t)kKcapMax * 4;
   s.st_vals = reinterpret_cast<float*>(p);
+  s.binlist = reinterpret_cast<Candidate*>(p);
   p += (size_t)kKcapMax * 4;
-  s.coarse = reinterpret_cast<uint32_t*>(p);
-  p += (size_t)kCoarseBins * 4;
-  s.fine = reinterpret_cast<uint32_t*>(p);
-  p += (size_t)kFineBins * 4;
-  s.sel = reinterpret_cast<uint32_t*>(p);
-  p += (size_t)kSelBins * 4;
+  s.hist = reinterpret_cast<uint32_t*>(p);
+  p += (size_t)kHistBins * 4;
+  s.masks = reinterpret_cast<uint32_t*>(p);
+  p += (size_t)mask_words * NF * 32 * 4;
   s.bitmap = reinterpret_cast<uint32_t*>(p);
   p += (size_t)vwords * 4;
-  s.binlist = reinterpret_cast<Candidate*>(p);
-  p += (size_t)kBinListCap * sizeof(Candidate);
   s.full = reinterpret_cast<uint64_t*>(p);
   s.empty = s.full + n_stages;
   s.cand_full = s.empty + n_stages;
-  s.cand_free = s.cand_full + 2;
+  s.cand_free = s.cand_full + 1;
   p += 32 * 8;
   s.scan_f = reinterpret_cast<uint64_t*>(p);
   p += (2 * 32 + 8) * 8;
   s.scan_p = reinterpret_cast<uint64_t*>(p);
   p += (2 * 32 + 8) * 8;
-  s.meta = reinterpret_cast<RowMeta*>(p);
-  p += 2 * sizeof(RowMeta);
   s.ctl = reinterpret_cast<int*>(p);
   p += kCtlWords * 4;
+  s.tile_of = reinterpret_cast<uint16_t*>(p);
+  p += (size_t)NF * kItersMax * 2;
   s.wprefix = reinterpret_cast<uint16_t*>(p);
   return s;
 }
@@ -305,10 +313,10 @@ __device__ __forceinline__ PipeSmem<NF> carve_pipe_smem(unsigned char* base, int
 // Largest bin b with (entries in bins > b) < target <= (entries in bins >= b).  The count above it goes
 // to ctl[c_bin + 1], the bin's own count to ctl[c_bin + 2]; ctl[c_bin] = -1 when the histogram holds
 // fewer than `target` entries.  All NT threads of the group call it; every bin is read by exactly one
-// thread, which leaves it zero for the next row.
+// thread, which leaves it zero for its next use.  Two barriers.
 template <int BINS, int NT, int BAR>
-__device__ __forceinline__ void find_rank_bin(uint32_t* hist, uint32_t target, int tid, uint64_t* scratch, int* ctl,
-                                              int c_bin) {
+__device__ __forceinline__ void find_rank_bin(uint32_t* hist, uint32_t target, int tid, uint64_t* scratch, int& flip,
+                                              int* ctl, int c_bin) {
   constexpr int PER = BINS / NT;
   static_assert(BINS % NT == 0 && PER % 4 == 0, "bins must split into 16-byte pieces per thread");
   // thread t owns bins BINS-1 - PER*t - j, j = 0..PER-1, i.e. words [BINS - PER (t+1), BINS - PER t)
@@ -322,9 +330,9 @@ __device__ __forceinline__ void find_rank_bin(uint32_t* hist, uint32_t target, i
   }
 #pragma unroll
   for (int j = 0; j < PER; ++j) sum += c[j];
-  if (tid == 0) ctl[c_bin] = -1;
+  if (tid == 0) ctl[c_bin] = -1;  // ordered before the owner's write by the barrier inside the scan
   uint32_t total;
-  uint32_t above = group_exclusive_scan<NT, BAR, uint32_t>(sum, tid, scratch, &total);
+  uint32_t above = group_scan1<NT, BAR, uint32_t>(sum, tid, scratch, flip, &total);
   if (above < target && target <= above + sum) {
 #pragma unroll
     for (int j = 0; j < PER; ++j) {
@@ -339,68 +347,55 @@ __device__ __forceinline__ void find_rank_bin(uint32_t* hist, uint32_t target, i
   group_sync<NT, BAR>();
 }
 
-// Visit the candidates of one row: finisher warp pw takes the lists of filter warps pw, pw+NP, ...;
-// four independent entries per lane are in flight at a time.
-template <int NF, int NP, typename F>
-__device__ __forceinline__ void for_each_candidate(const Candidate* lists, const int* count, int pw, int lane, F f) {
-  for (int seg = pw; seg < NF; seg += NP) {
-    const Candidate* s = lists + (size_t)seg * kWarpListCap;
-    const int n = min(count[seg], kWarpListCap);
-    for (int i0 = 0; i0 < n; i0 += 128) {
-      Candidate c[4];
-      bool v[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int i = i0 + q * 32 + lane;
-        v[q] = i < n;
-        if (v[q]) c[q] = s[i];
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        if (v[q]) f(c[q]);
-    }
-  }
+// float of an order-preserving key (inverse of float_key)
+__device__ __forceinline__ float key_float(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
 template <int DTYPE, int NF, int NP>
 __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(const RowArgs a, const PipeCfg cfg) {
   constexpr int NT_F = NF * 32, NT_P = NP * 32;
   constexpr int BAR_F = 1, BAR_P = 2;
+  constexpr uint32_t kStride = NT_F * 8;  // bytes between consecutive entries of one filter thread
   static_assert(NF <= 16 && NP * 32 * kFinItems >= kKcapMax, "group sizes");
   using TR = PipeTraits<DTYPE>;
   constexpr int TPS = TR::kTilesPerStage;
   extern __shared__ unsigned char smem_raw[];
-  PipeSmem<NF> sm = carve_pipe_smem<NF>(smem_raw, cfg.n_stages, cfg.vwords);
+  PipeSmem<NF> sm = carve_pipe_smem<NF>(smem_raw, cfg.n_stages, cfg.vwords, cfg.mask_words);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int NS = cfg.n_stages;
   const bool has_u = a.uncond != nullptr;
   const float neg_inf = __int_as_float(0xff800000);
+  const float lowest = -3.402823466e38f;  // with this threshold every finite value is a candidate
 
-  // ---- one-time set-up: barriers and the tables that must start at zero ----
+  const RowSchedule sched(a.V, cfg.sample_stride, TPS);
+  const int rows = a.B * a.W;
+  const int mask_words = cfg.mask_words;
+
+  // ---- one-time set-up: barriers, the tables that must start at zero, the tile map ----
   if (threadIdx.x == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(&sm.full[s], 1);
       mbar_init(&sm.empty[s], NF);
     }
-    for (int k = 0; k < 2; ++k) {
-      mbar_init(&sm.cand_full[k], NF);
-      mbar_init(&sm.cand_free[k], 1);
-    }
+    mbar_init(sm.cand_full, NF);
+    mbar_init(sm.cand_free, 1);
     for (int k = 0; k < kCtlWords; ++k) sm.ctl[k] = 0;
     fence_barrier_init();
   }
-  for (int j = threadIdx.x; j < kCoarseBins; j += blockDim.x) sm.coarse[j] = 0;
-  for (int j = threadIdx.x; j < kFineBins; j += blockDim.x) sm.fine[j] = 0;
+  for (int j = threadIdx.x; j < kHistBins; j += blockDim.x) sm.hist[j] = 0;
   for (int j = threadIdx.x; j < kSelBins; j += blockDim.x) sm.sel[j] = 0;
   for (int j = threadIdx.x; j < cfg.vwords; j += blockDim.x) sm.bitmap[j] = 0;
-  if (threadIdx.x < 32) {
-    sm.meta[0].count[threadIdx.x & 15] = 0;
-    sm.meta[1].count[threadIdx.x & 15] = 0;
+  if (warp < NF && lane == 0) {
+    int it = 0;
+    for (int s = 0; s < sched.stages; ++s) {
+      const int nt = sched.stage_tiles(s, TPS);
+      for (int j = warp; j < nt; j += NF)
+        if (it < kItersMax) sm.tile_of[warp * kItersMax + it++] = (uint16_t)sched.global_tile(s, j, TPS);
+    }
   }
   __syncthreads();
 
-  const RowSchedule sched(a.V, cfg.sample_stride, TPS);
-  const int rows = a.B * a.W;
   volatile int* abort_flag = sm.ctl + kCtlAbort;
 
   if (warp == NF + NP) {
@@ -475,7 +470,9 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
     const int fw = warp;
     const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
     const bool has_t = a.inv_T != 1.0f;
-    int slot = 0;
+    const uint32_t list_base = smem_u32(sm.ylist) + (uint32_t)tid * 8u;
+    const uint32_t list_limit = list_base + (uint32_t)(kListCap - 4) * kStride;  // beyond it a tile may not fit
+    int slot = 0, flip = 0;
     uint32_t phase = 0;
     uint32_t n_row = 0;
     bool dead = false;
@@ -483,13 +480,10 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       const int b = row / a.W, i = row - b * a.W;
       const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
       if (i >= L || dead) continue;
-      const int buf = (int)(n_row & 1u);
-      const uint32_t buf_use = n_row >> 1;
-      RowMeta* meta = sm.meta + buf;
-      Candidate* seg = sm.lists + ((size_t)buf * NF + fw) * kWarpListCap;
 
-      // ---------------- sample stages: histogram of the order-preserving keys ----------------
+      // ---------------- sample, pass A: maxima of groups of eight, by key ----------------
       bool ok = true;
+      float smax = neg_inf;
       {
         int sl = slot;
         uint32_t ph = phase;
@@ -503,8 +497,9 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
               float y[8];
               tile_y8<DTYPE>(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes, has_u, has_t, lane, s2,
                              t2, y);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) atomicAdd(&sm.coarse[float_key(canonical(y[e])) >> 21], 1u);
+              const float m8 = max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]);
+              atomicAdd(&sm.hist[float_key(canonical(m8)) >> 21], 1u);
+              smax = fmaxf(smax, m8);
             }
           }
           if (++sl == NS) {
@@ -513,16 +508,26 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
           }
         }
       }
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, d));
+      if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(&sm.ctl[kCtlSmaxKey]), float_key(canonical(smax)));
       dead = group_any<NT_F, BAR_F>(!ok);
       if (dead) {
         if (tid == 0) *abort_flag = 1;
         continue;
       }
-      find_rank_bin<kCoarseBins, NT_F, BAR_F>(sm.coarse, (uint32_t)cfg.sample_rank, tid, sm.scan_f, sm.ctl, kCtlFBin);
+      // at least m group maxima, hence at least m sample elements, are >= the lower edge of this bin
+      find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kCtlFBin);
       const int cbin = sm.ctl[kCtlFBin];
-      const int fine_target = cfg.sample_rank - sm.ctl[kCtlFAbove];
-      // ---------------- second level inside the coarse bin ----------------
-      {
+      float floor_y = cbin >= 0 ? key_float((uint32_t)cbin << 21) : lowest;
+      if (!(floor_y >= lowest)) floor_y = lowest;  // edge fell on -inf or into the NaN patterns
+      const float top_y = key_float((uint32_t)sm.ctl[kCtlSmaxKey]);
+      const bool refine = floor_y > lowest && top_y >= floor_y && top_y <= 3.402823466e38f;
+      const float range = __fsub_rn(top_y, floor_y);
+      const float scale = (refine && range > 0.0f) ? __fdiv_rn((float)kHistBins - 0.5f, range) : 0.0f;
+      float tau0 = lowest;
+      if (refine) {
+        // ---------------- sample, pass B: linear bins over [floor, sample max] ----------------
         int sl = slot;
         for (int s = 0; s < sched.sample_stages; ++s) {
           const unsigned char* st_c = sm.ring + (size_t)sl * TR::kStageBytes;
@@ -534,76 +539,64 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
                            y);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-              const uint32_t k = float_key(canonical(y[e]));
-              if ((int)(k >> 21) == cbin) atomicAdd(&sm.fine[(k >> 13) & 0xffu], 1u);
+              if (y[e] >= floor_y) {
+                const int q = __float2int_rd(__fmul_rn(__fsub_rn(y[e], floor_y), scale));
+                atomicAdd(&sm.hist[min(max(q, 0), kHistBins - 1)], 1u);
+              }
             }
           }
           if (++sl == NS) sl = 0;
         }
+        group_sync<NT_F, BAR_F>();
+        find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kCtlFBin);
+        const int fbin = sm.ctl[kCtlFBin];
+        if (fbin > 0 && scale > 0.0f) {
+          // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
+          const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
+          tau0 = __fadd_rd(floor_y, t);
+        } else if (fbin == 0 || (fbin > 0 && scale == 0.0f)) {
+          tau0 = floor_y;
+        }
       }
-      group_sync<NT_F, BAR_F>();
-      if (fw == 0) {
-        // lane l owns fine bins 255-8l .. 248-8l; walk from the largest bin down
-        uint32_t c[8], sum = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          c[j] = sm.fine[255 - 8 * lane - j];
-          sm.fine[255 - 8 * lane - j] = 0;
-          sum += c[j];
-        }
-        uint32_t inc = sum;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          const uint32_t n = __shfl_up_sync(0xffffffffu, inc, d);
-          if (lane >= d) inc += n;
-        }
-        uint32_t above = inc - sum;
-        const uint32_t target = (uint32_t)fine_target;
-        int fbin = -1;
-        if (above < target && target <= inc) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if (above < target && target <= above + c[j]) fbin = 255 - 8 * lane - j;
-            above += c[j];
-          }
-        }
-        const float lowest = -3.402823466e38f;  // with this threshold every finite value is a candidate
-        const bool found = fbin >= 0 && cbin >= 0;
-        if (found) {
-          // lower edge of (coarse bin, fine bin) as a float: every value of the bin is >= it
-          const uint32_t key = ((uint32_t)cbin << 21) | ((uint32_t)fbin << 13);
-          const uint32_t bits = (key & 0x80000000u) ? (key & 0x7fffffffu) : ~key;
-          float t0 = __uint_as_float(bits);
-          if (!(t0 >= lowest)) t0 = lowest;  // edge fell on -inf or into the NaN patterns
-          sm.ctl[kCtlTau0] = __float_as_int(t0);
-        }
-        if (!__any_sync(0xffffffffu, found) && lane == 0) sm.ctl[kCtlTau0] = __float_as_int(lowest);
-      }
-      // ---------------- the candidate buffer must be back from the finisher ----------------
-      if (buf_use > 0) ok = mbar_wait(&sm.cand_free[buf], (buf_use - 1) & 1u);
-      dead = group_any<NT_F, BAR_F>(!ok);  // also publishes tau0
+      // ---------------- lists and hit bits must be back from the finisher ----------------
+      if (n_row > 0) ok = mbar_wait(sm.cand_free, (n_row - 1) & 1u);
+      dead = group_any<NT_F, BAR_F>(!ok);
       if (dead) {
         if (tid == 0) *abort_flag = 1;
         continue;
       }
-      const float tau0 = __int_as_float(sm.ctl[kCtlTau0]);
-      int* wcount = &meta->count[fw];
-      if (lane == 0) *wcount = 0;
-      __syncwarp();
-      float vmax = neg_inf;
-      auto filter_tile = [&](const unsigned char* ctile, const unsigned char* utile, int id_base) {
+      if (tid == 0) sm.ctl[kCtlSmaxKey] = 0;  // every thread has read it; next written after the next row's barriers
+
+      uint32_t cur = list_base;  // shared-memory address of the thread's next free entry
+      uint32_t imw = 0;          // inverted hit bits of the last (it & 7) tiles
+      int it = 0;                // tiles this warp has filtered in this row
+      bool overflow = false;
+      // One tile: four pairs.  Pair k is stored at cur + k*stride minus one stride for every earlier miss
+      // of this tile; z < 0 (sign bit set) marks a miss.  A pair of NaNs counts as a hit and is dropped
+      // later; -inf never hits.
+      auto filter_tile = [&](const unsigned char* ctile, const unsigned char* utile) {
         float y[8];
         tile_y8<DTYPE>(ctile, utile, has_u, has_t, lane, s2, t2, y);
-        vmax = max3(vmax, y[0], y[1]);
-        vmax = max3(vmax, y[2], y[3]);
-        vmax = max3(vmax, y[4], y[5]);
-        vmax = max3(vmax, y[6], y[7]);
+        if (cur > list_limit) {
+          overflow = true;
+          cur = list_base;
+        }
+        uint32_t d = cur;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          if (y[e] >= tau0) {
-            const int pos = atomicAdd(wcount, 1);
-            if (pos < kWarpListCap) seg[pos] = Candidate{y[e], id_base + tile_elem<DTYPE>(lane, e)};
-          }
+        for (int k = 0; k < 4; ++k) {
+          const float m = fmaxf(y[2 * k], y[2 * k + 1]);
+          const uint32_t miss = __umulhi(__float_as_uint(__fsub_rn(m, tau0)), 2u);
+          asm volatile("st.shared.v2.f32 [%0+%3], {%1, %2};" ::"r"(d), "f"(y[2 * k]), "f"(y[2 * k + 1]),
+                       "n"(0)
+                       : "memory");
+          d = d + kStride - miss * kStride;
+          imw = imw * 2u + miss;
+        }
+        cur = d;
+        ++it;
+        if ((it & 7) == 0) {
+          if ((it >> 3) <= mask_words) sm.masks[(size_t)((it >> 3) - 1) * NT_F + tid] = imw;
+          imw = 0;
         }
       };
       // ---------------- the sample tiles, now against tau0 ----------------
@@ -611,9 +604,7 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
         const unsigned char* st_c = sm.ring + (size_t)slot * TR::kStageBytes;
         const unsigned char* st_u = st_c + kStageArrayBytes;
         const int nt = sched.stage_tiles(s, TPS);
-        for (int j = fw; j < nt; j += NF)
-          filter_tile(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes,
-                      sched.global_tile(s, j, TPS) * kTileElems);
+        for (int j = fw; j < nt; j += NF) filter_tile(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes);
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.empty[slot]);
         if (++slot == NS) {
@@ -628,9 +619,7 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
           const unsigned char* st_c = sm.ring + (size_t)slot * TR::kStageBytes;
           const unsigned char* st_u = st_c + kStageArrayBytes;
           const int nt = sched.stage_tiles(s, TPS);
-          for (int j = fw; j < nt; j += NF)
-            filter_tile(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes,
-                        sched.global_tile(s, j, TPS) * kTileElems);
+          for (int j = fw; j < nt; j += NF) filter_tile(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.empty[slot]);
@@ -639,18 +628,25 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
           phase ^= 1u;
         }
       }
-#pragma unroll
-      for (int d = 16; d > 0; d >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, d));
-      if (lane == 0) {
-        meta->vmax[fw] = vmax;
-        if (fw == 0) meta->tau0 = tau0;
+      // ---------------- hand the row over ----------------
+      {
+        const int rem = it & 7;
+        int w = it >> 3;
+        if (rem != 0 && w < mask_words) {
+          const int fill = 32 - 4 * rem;  // bits of the word not reached: misses
+          sm.masks[(size_t)w * NT_F + tid] = (imw << fill) | ((1u << fill) - 1u);
+          ++w;
+        }
+        for (; w < mask_words; ++w) sm.masks[(size_t)w * NT_F + tid] = 0xffffffffu;
+        if (overflow) sm.ctl[kCtlRowOverflow] = 1;
+        if (tid == 0) sm.ctl[kCtlRowTau0] = __float_as_int(tau0);
       }
       dead = group_any<NT_F, BAR_F>(!ok);
       if (dead) {
         if (tid == 0) *abort_flag = 1;
-        continue;  // the buffer is not handed over: the finisher's wait runs out and marks the rows
+        continue;  // the row is not handed over: the finisher's wait runs out and marks the rows
       }
-      if (lane == 0) mbar_arrive(&sm.cand_full[buf]);
+      if (lane == 0) mbar_arrive(sm.cand_full);
       ++n_row;
     }
     return;
@@ -658,7 +654,7 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
 
   // ======================================= finisher warps =======================================
   const int tid = threadIdx.x - NT_F;  // 0 .. NT_P-1
-  const int pw = tid >> 5;
+  int flip = 0;
   uint32_t n_row = 0;
   bool dead = false;
   for (int row = blockIdx.x; row < rows; row += gridDim.x) {
@@ -673,9 +669,13 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       continue;
     }
     const int kcap = a.kcap;
-    const int buf = (int)(n_row & 1u);
     const int draft = a.drafts ? a.drafts[row] : -1;
-    if (!dead) dead = !mbar_wait(&sm.cand_full[buf], (n_row >> 1) & 1u);
+    // the row's own random number: needed last, computed while waiting
+    const int pos = (a.pos_base ? a.pos_base[b] : 0) + i;
+    const int iter = a.iteration ? a.iteration[b] : a.iteration0;
+    const Philox4 rnd = philox4x32_10((uint32_t)pos, (uint32_t)(a.seq_base + b), (uint32_t)iter, (uint32_t)a.purpose,
+                                      a.seed_lo, a.seed_hi);
+    if (!dead) dead = !mbar_wait(sm.cand_full, n_row & 1u);
     dead = group_any<NT_P, BAR_P>(dead || (*abort_flag != 0));
     if (dead) {
       if (tid == 0) {
@@ -685,22 +685,81 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       }
       continue;
     }
-    const RowMeta* meta = sm.meta + buf;
-    const Candidate* lists = sm.lists + (size_t)buf * NF * kWarpListCap;
-    const float tau0 = meta->tau0;
-    int n_total = 0;
-    bool fallback = kcap > kKcapMax;
-    float vmax = neg_inf;
-#pragma unroll
-    for (int w = 0; w < NF; ++w) {
-      const int c = meta->count[w];
-      fallback |= c > kWarpListCap;
-      n_total += c;
-      vmax = fmaxf(vmax, meta->vmax[w]);
+    const float tau0 = __int_as_float(sm.ctl[kCtlRowTau0]);
+    bool fallback = kcap > kKcapMax || sm.ctl[kCtlRowOverflow] != 0;
+
+    // ---- lists + hit bits -> dense candidate list.  Pass 1 counts the values that reach tau0 ----
+    uint32_t my_valid = 0;
+    if (!fallback) {
+      for (int col = tid; col < NT_F; col += NT_P) {
+        int n_e = 0;
+        for (int w = 0; w < mask_words; ++w) n_e += __popc(~sm.masks[(size_t)w * NT_F + col]);
+        n_e = min(n_e, kListCap);
+        for (int e = 0; e < n_e; ++e) {
+          const float2 pr = *reinterpret_cast<const float2*>(&sm.ylist[(size_t)e * NT_F + col]);
+          my_valid += (pr.x >= tau0 ? 1u : 0u) + (pr.y >= tau0 ? 1u : 0u);
+        }
+      }
     }
-    fallback |= n_total < kcap;
+    uint32_t n_total;
+    uint32_t my_off = group_scan1<NT_P, BAR_P, uint32_t>(my_valid, tid, sm.scan_p, flip, &n_total);
+    fallback |= n_total < (uint32_t)kcap || n_total > (uint32_t)kDenseCap;
+    // ---- pass 2 decodes the token ids from the hit bits and writes the dense list ----
+    float vmax = neg_inf;
+    if (!fallback) {
+      for (int col = tid; col < NT_F; col += NT_P) {
+        const int cw = col >> 5, cl = col & 31;
+        int e = 0;
+        for (int w = 0; w < mask_words; ++w) {
+          uint32_t x = ~sm.masks[(size_t)w * NT_F + col];
+          while (x != 0u && e < kListCap) {
+            const int bitpos = __clz((int)x);
+            x &= ~(0x80000000u >> bitpos);
+            const int q = w * 32 + bitpos;  // pair index within the row for this thread
+            const int tile = sm.tile_of[cw * kItersMax + (q >> 2)];
+            const int id = tile * kTileElems + tile_elem<DTYPE>(cl, 2 * (q & 3));
+            const float2 pr = *reinterpret_cast<const float2*>(&sm.ylist[(size_t)e * NT_F + col]);
+            ++e;
+            if (pr.x >= tau0) {
+              sm.dense[my_off++] = Candidate{pr.x, id};
+              vmax = fmaxf(vmax, pr.x);
+            }
+            if (pr.y >= tau0) {
+              sm.dense[my_off++] = Candidate{pr.y, id + 1};
+              vmax = fmaxf(vmax, pr.y);
+            }
+          }
+        }
+      }
+    }
+    vmax = group_max1_f32<NT_P, BAR_P>(vmax, tid, sm.scan_p, flip);
+    // lists and hit bits are not read again: hand them back
+    if (tid == 0) {
+      sm.ctl[kCtlRowOverflow] = 0;
+      sm.ctl[kCtlGather] = 0;
+      sm.ctl[kCtlPtok] = 0;
+      sm.ctl[kCtlFoundId] = -1;
+      mbar_arrive(sm.cand_free);
+    }
+    ++n_row;
     fallback |= !(vmax <= 3.402823466e38f);  // an infinite logit: the any-shape path decides what the row is
 
+    // visit the dense list, four independent entries per thread in flight
+    auto for_each_candidate = [&](auto f) {
+      for (uint32_t i0 = 0; i0 < n_total; i0 += 4 * NT_P) {
+        Candidate c[4];
+        bool v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t ix = i0 + q * NT_P + tid;
+          v[q] = ix < n_total;
+          if (v[q]) c[q] = sm.dense[ix];
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (v[q]) f(c[q]);
+      }
+    };
     int tbin = 0, need = 0, nbin = 0;
     const float range = __fsub_rn(vmax, tau0);
     const float scale = range > 0.0f ? __fdiv_rn((float)kSelBins * 0.999f, range) : 0.0f;
@@ -710,22 +769,20 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       return min(max(q, 0), kSelBins - 1);
     };
     if (!fallback) {
-      for_each_candidate<NF, NP>(lists, meta->count, pw, lane,
-                                 [&](const Candidate& c) { atomicAdd(&sm.sel[bin_of(c.y)], 1u); });
+      for_each_candidate([&](const Candidate& c) { atomicAdd(&sm.sel[bin_of(c.y)], 1u); });
       group_sync<NT_P, BAR_P>();
-      find_rank_bin<kSelBins, NT_P, BAR_P>(sm.sel, (uint32_t)kcap, tid, sm.scan_p, sm.ctl, kCtlPBin);
+      find_rank_bin<kSelBins, NT_P, BAR_P>(sm.sel, (uint32_t)kcap, tid, sm.scan_p, flip, sm.ctl, kCtlPBin);
       tbin = sm.ctl[kCtlPBin];
       need = kcap - sm.ctl[kCtlPAbove];  // members of the threshold bin that survive
       nbin = sm.ctl[kCtlPCount];
       if (tbin < 0 || nbin > kBinListCap) fallback = true;
     }
-    uint32_t wsum = 0, wrun = 0;
     const int wper = (cfg.vwords + NT_P - 1) / NT_P;
     const int w0 = min(tid * wper, cfg.vwords), w1 = min(w0 + wper, cfg.vwords);
     if (!fallback) {
       // ---- survivors into the bitmap over token ids: everything above the threshold bin, and the
       //      `need` best of the bin itself by (y descending, id ascending) ----
-      for_each_candidate<NF, NP>(lists, meta->count, pw, lane, [&](const Candidate& c) {
+      for_each_candidate([&](const Candidate& c) {
         const int q = bin_of(c.y);
         if (q > tbin) atomicOr(&sm.bitmap[c.id >> 5], 1u << (c.id & 31));
         else if (q == tbin) sm.binlist[atomicAdd(&sm.ctl[kCtlGather], 1)] = Candidate{canonical(c.y), c.id};
@@ -742,9 +799,10 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       }
       group_sync<NT_P, BAR_P>();
       // ---- exclusive prefix of the per-word popcounts; each thread owns a contiguous run of words ----
+      uint32_t wsum = 0;
       for (int w = w0; w < w1; ++w) wsum += __popc(sm.bitmap[w]);
       uint32_t total;
-      wrun = group_exclusive_scan<NT_P, BAR_P, uint32_t>(wsum, tid, sm.scan_p, &total);
+      uint32_t wrun = group_scan1<NT_P, BAR_P, uint32_t>(wsum, tid, sm.scan_p, flip, &total);
       for (int w = w0; w < w1; ++w) {
         sm.wprefix[w] = (uint16_t)wrun;
         wrun += __popc(sm.bitmap[w]);
@@ -753,31 +811,23 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       group_sync<NT_P, BAR_P>();
     }
     if (!fallback) {
-      // ---- softmax numerators into ascending-id order ----
-      for_each_candidate<NF, NP>(lists, meta->count, pw, lane, [&](const Candidate& c) {
+      // ---- softmax numerators into ascending-id order (this overwrites sel and binlist) ----
+      for_each_candidate([&](const Candidate& c) {
         const uint32_t w = sm.bitmap[c.id >> 5];
         const uint32_t bit = 1u << (c.id & 31);
         if (w & bit) {
-          const int pos = (int)sm.wprefix[c.id >> 5] + __popc(w & (bit - 1u));
-          sm.st_ids[pos] = c.id;
-          sm.st_vals[pos] = exp_diff(canonical(c.y), vmax);
+          const int p = (int)sm.wprefix[c.id >> 5] + __popc(w & (bit - 1u));
+          sm.st_ids[p] = c.id;
+          sm.st_vals[p] = exp_diff(canonical(c.y), vmax);
         }
       });
     }
     group_sync<NT_P, BAR_P>();
-    // the candidate lists are not read again: hand the buffer back, leave the tables clean
-    if (tid == 0) {
-      mbar_arrive(&sm.cand_free[buf]);
-      sm.ctl[kCtlGather] = 0;
-      sm.ctl[kCtlPtok] = 0;
-      sm.ctl[kCtlFoundId] = -1;
-    }
-    ++n_row;
     for (int w = w0; w < w1; ++w) sm.bitmap[w] = 0;
     if (fallback) {
-      // exact any-shape path from global memory (the row is still in L2)
-      group_sync<NT_P, BAR_P>();
-      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_ids));
+      // exact any-shape path from global memory (the row is still in L2); its scratch sits on st_vals,
+      // so that sel (= st_ids) stays zero
+      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals));
       continue;
     }
     // ---- normalise, write the row, draw from it ----
@@ -792,7 +842,12 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       ids[j] = in ? sm.st_ids[k0 + j] : -1;
       zpart += e[j];
     }
-    const float Z = group_sum_f32<NT_P, BAR_P>(zpart, tid, sm.scan_p);
+    // these eight words of st_ids are this thread's share of sel: zero again for the next row
+    if (k0 + kFinItems <= kSelBins) {
+      *reinterpret_cast<uint4*>(sm.sel + k0) = make_uint4(0u, 0u, 0u, 0u);
+      *reinterpret_cast<uint4*>(sm.sel + k0 + 4) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    const float Z = group_sum1_f32<NT_P, BAR_P>(zpart, tid, sm.scan_p, flip);
     int32_t* out_ids = a.out_ids + (size_t)row * kcap;
     float* out_vals = a.out_vals + (size_t)row * kcap;
     uint64_t wgt[kFinItems], wloc = 0;
@@ -821,12 +876,8 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       }
     }
     // the row's own draw from p_i: fixed-point inverse CDF in ascending-id order
-    const int pos = (a.pos_base ? a.pos_base[b] : 0) + i;
-    const int iter = a.iteration ? a.iteration[b] : a.iteration0;
-    const Philox4 rnd = philox4x32_10((uint32_t)pos, (uint32_t)(a.seq_base + b), (uint32_t)iter, (uint32_t)a.purpose,
-                                      a.seed_lo, a.seed_hi);
     uint64_t T;
-    const uint64_t lo = group_exclusive_scan<NT_P, BAR_P, uint64_t>(wloc, tid, sm.scan_p, &T);
+    const uint64_t lo = group_scan1<NT_P, BAR_P, uint64_t>(wloc, tid, sm.scan_p, flip, &T);
     const uint64_t t = __umul64hi(random64(rnd), T);
     if (T > 0 && t >= lo && t < lo + wloc) {
       uint64_t run = lo;

@@ -27,7 +27,7 @@ int cuda_fail(cudaError_t e, const char* what) {
 }
 
 constexpr int kGenericThreads = 512;
-constexpr int kVerifyThreads = 256;
+constexpr int kVerifyThreads = 512;
 
 int sm_count() {
   static int cached = 0;
@@ -49,10 +49,11 @@ constexpr size_t kSmemLimit = 227u * 1024u;
 
 // Decide whether the single-pass pipelined kernel can take this shape, and with which sampling
 // parameters.  The sample is every SS-th 256-element tile of a row; its rank-m value (from the top)
-// becomes the candidate threshold.  m is chosen 4.5 standard deviations above K/SS, so that a row with
-// exchangeable entries fails to deliver K candidates with probability below 1e-5 (such a row is redone
-// by the any-shape path, never answered wrongly), and the candidate lists must hold the expected count
-// six standard deviations above its mean.
+// becomes the candidate threshold.  m is chosen 3.5 standard deviations above K/SS, so that a row with
+// exchangeable entries fails to deliver K candidates with probability below 3e-4 (such a row is redone
+// by the any-shape path, never answered wrongly).  The on-chip lists must hold the expected number of
+// candidates with a margin: four standard deviations for the row's total, and for the share of one
+// filter thread (a Poisson count) a tail below 1e-6.
 bool plan_pipeline(const sjd_params* P, int kcap, sjd::PipeCfg* cfg, size_t* smem) {
   const int V = P->V;
   if (kcap > sjd::kKcapMax || V % sjd::kTileElems != 0) return false;
@@ -60,27 +61,36 @@ bool plan_pipeline(const sjd_params* P, int kcap, sjd::PipeCfg* cfg, size_t* sme
   const int tps = sjd::kStageArrayBytes / tile_bytes;
   const int tiles = V / sjd::kTileElems;
   const int vwords = V / 32;
-  const size_t fixed = sjd::pipe_smem_fixed_bytes(kFilterWarps, vwords);
-  if (fixed + 4 * 2 * (size_t)sjd::kStageArrayBytes > kSmemLimit) return false;
-  int ns = (int)((kSmemLimit - fixed) / (2 * (size_t)sjd::kStageArrayBytes));
-  if (ns > kMaxStages) ns = kMaxStages;
+  if (tiles > sjd::kItersMax * kFilterWarps) return false;
   for (int ss : {8, 16, 32}) {
     if (tiles % ss != 0) continue;
-    const int sample_tiles = tiles / ss;
+    const int sample_tiles = tiles / ss, tail_tiles = tiles - sample_tiles;
     const int sample_stages = (sample_tiles + tps - 1) / tps;
-    if (sample_stages + 3 > ns) continue;
+    // tiles of filter warp 0 per row (the most any warp gets), four hit bits each
+    int iters0 = 0;
+    for (int left = sample_tiles; left > 0; left -= tps) iters0 += ((left < tps ? left : tps) + kFilterWarps - 1) / kFilterWarps;
+    for (int left = tail_tiles; left > 0; left -= tps) iters0 += ((left < tps ? left : tps) + kFilterWarps - 1) / kFilterWarps;
+    const int mask_words = (4 * iters0 + 31) / 32;
+    if (iters0 > sjd::kItersMax || mask_words > sjd::kMaskWordsMax) continue;
+    const size_t fixed = sjd::pipe_smem_fixed_bytes(kFilterWarps, vwords, mask_words);
+    if (fixed + (size_t)(sample_stages + 3) * 2 * sjd::kStageArrayBytes > kSmemLimit) continue;
+    int ns = (int)((kSmemLimit - fixed) / (2 * (size_t)sjd::kStageArrayBytes));
+    if (ns > kMaxStages) ns = kMaxStages;
     const int n_sample = V / ss;
     const double a = (double)kcap / ss;
-    const double root = 2.25 + std::sqrt(2.25 * 2.25 + a);
+    const double root = 1.75 + std::sqrt(1.75 * 1.75 + a);
     const int m = (int)std::ceil(root * root);
-    if (m > n_sample / 2) continue;
-    const double expect = ((double)m + 6.0 * std::sqrt((double)m)) * ss;
-    if (expect > 0.9 * (double)sjd::kWarpListCap * kFilterWarps) continue;
+    if (m > n_sample / 2 || m > 32 * sample_tiles) continue;  // the rank must exist among the group maxima too
+    const double mean = (double)m * ss, sd = (double)ss * std::sqrt((double)m);
+    if (mean + 4.0 * sd > (double)sjd::kDenseCap) continue;
+    const double per_thread = mean / (32.0 * kFilterWarps);
+    if (per_thread + 5.5 * std::sqrt(per_thread) + 1.0 > (double)(sjd::kListCap - 4)) continue;
     cfg->sample_stride = ss;
     cfg->sample_rank = m;
     cfg->n_stages = ns;
     cfg->vwords = vwords;
-    *smem = sjd::pipe_smem_bytes(ns, kFilterWarps, vwords);
+    cfg->mask_words = mask_words;
+    *smem = sjd::pipe_smem_bytes(ns, kFilterWarps, vwords, mask_words);
     return true;
   }
   return false;

@@ -64,8 +64,12 @@ __device__ __forceinline__ float likelihood_ratio(float p, float q) {
   return __fdiv_rn(p, q);
 }
 
+constexpr int kVerifyStageCap = 2048;  // entries of a previous-iteration row staged in shared memory
+
 struct VerifySmem {
   uint64_t scan[2 * 32 + 8];
+  int32_t q_ids[kVerifyStageCap];
+  float q_vals[kVerifyStageCap];
   int first_reject;
   int status;
   int res_tok;
@@ -82,6 +86,7 @@ __device__ void verify_sequence(const VerifyArgs& a, int b, int tid, VerifySmem&
   const bool draft_all = (a.flags & kFlagDraftAll) != 0;
   const bool reuse_on = (a.flags & kFlagReuse) != 0;
   const size_t base = (size_t)b * W;
+  int flip = 0;
   if (tid == 0) {
     sm.first_reject = L;
     sm.status = 0;
@@ -99,8 +104,8 @@ __device__ void verify_sequence(const VerifyArgs& a, int b, int tid, VerifySmem&
     if (!draft_all) {
       const float q = a.q_tok[base + i];
       const float ratio = likelihood_ratio(rs.p_tok, q);
-      const Philox4 rnd = philox4x32_10((uint32_t)(pos0 + i), (uint32_t)(a.seq_base + b), (uint32_t)iter, kPurposeAccept, a.seed_lo,
-                                        a.seed_hi);
+      const Philox4 rnd = philox4x32_10((uint32_t)(pos0 + i), (uint32_t)(a.seq_base + b), (uint32_t)iter, kPurposeAccept,
+                                        a.seed_lo, a.seed_hi);
       const float u = uniform24(rnd.x0);
       if (!(u < fminf(ratio, 1.0f))) atomicMin(&sm.first_reject, i);
       if (!(q > 0.0f)) st |= kStatusQtok;
@@ -110,30 +115,75 @@ __device__ void verify_sequence(const VerifyArgs& a, int b, int tid, VerifySmem&
   group_sync<NT, BAR>();
   const int acc = draft_all ? 0 : sm.first_reject;
 
-  // Step 4, first rejected row: draw from max(0, p - q) / sum max(0, p - q)
+  // Step 4, first rejected row: draw from max(0, p - q) / sum max(0, p - q).  Every thread owns a run of
+  // consecutive entries of p_a (ascending token id), so one scan of the per-thread sums locates the draw.
   if (!draft_all && acc < L) {
     const size_t r = base + acc;
-    const int32_t* pid = a.p_ids + r * a.kcap;
-    const float* pv = a.p_vals + r * a.kcap;
-    const int32_t* qid = a.q_ids + r * a.kcap;
-    const float* qv = a.q_vals + r * a.kcap;
+    const int kcap = a.kcap;
+    const int32_t* pid = a.p_ids + r * kcap;
+    const float* pv = a.p_vals + r * kcap;
+    const int32_t* qid = a.q_ids + r * kcap;
+    const float* qv = a.q_vals + r * kcap;
     const int qc = a.q_cnt[r];
-    const float q_uniform = __fdiv_rn(1.0f, (float)a.V);
-    const Philox4 rnd = philox4x32_10((uint32_t)(pos0 + acc), (uint32_t)(a.seq_base + b), (uint32_t)iter, kPurposeResidual,
-                                      a.seed_lo, a.seed_hi);
-    auto residual = [&](int k) {
-      const float q = (qc == kQUniform) ? q_uniform : sparse_lookup(qid, qv, qc, pid[k]);
-      return fixed_weight(__fsub_rn(pv[k], q));
-    };
-    int k = group_icdf<NT, BAR>(residual, a.kcap, random64(rnd), tid, sm.scan);
-    if (k < 0) {  // no mass left after rounding: draw from p itself
-      if (tid == 0) sm.status |= kStatusEmptyResidual;
-      k = group_icdf<NT, BAR>([&](int kk) { return fixed_weight(pv[kk]); }, a.kcap, random64(rnd), tid, sm.scan);
-      if (k < 0) k = 0;
+    const bool staged = qc > 0 && qc <= kVerifyStageCap;
+    if (staged) {
+      for (int k = tid; k < qc; k += NT) {
+        sm.q_ids[k] = qid[k];
+        sm.q_vals[k] = qv[k];
+      }
+      group_sync<NT, BAR>();
     }
-    if (tid == 0) {
-      sm.res_tok = pid[k];
-      sm.res_prob = pv[k];
+    const int32_t* sid = staged ? sm.q_ids : qid;
+    const float* sval = staged ? sm.q_vals : qv;
+    const float q_uniform = __fdiv_rn(1.0f, (float)a.V);
+    const Philox4 rnd = philox4x32_10((uint32_t)(pos0 + acc), (uint32_t)(a.seq_base + b), (uint32_t)iter,
+                                      kPurposeResidual, a.seed_lo, a.seed_hi);
+    const uint64_t R = random64(rnd);
+    const int per = (kcap + NT - 1) / NT;
+    const int k0 = min(tid * per, kcap), k1 = min(k0 + per, kcap);
+    int found = -1;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      // attempt 0: residual weights; attempt 1 (only when they sum to zero after rounding): p itself
+      uint64_t local = 0;
+      for (int k = k0; k < k1; ++k) {
+        float w = pv[k];
+        if (attempt == 0) {
+          const float q = (qc == kQUniform) ? q_uniform : sparse_lookup(sid, sval, max(qc, 0), pid[k]);
+          w = __fsub_rn(w, q);
+        }
+        local += fixed_weight(w);
+      }
+      uint64_t T;
+      const uint64_t lo = group_scan1<NT, BAR, uint64_t>(local, tid, sm.scan, flip, &T);
+      if (T == 0) {
+        if (attempt == 0) {
+          if (tid == 0) sm.status |= kStatusEmptyResidual;
+          continue;
+        }
+        if (tid == 0) found = 0;
+        break;
+      }
+      const uint64_t t = __umul64hi(R, T);
+      if (t >= lo && t < lo + local) {
+        uint64_t run = lo;
+        for (int k = k0; k < k1; ++k) {
+          float w = pv[k];
+          if (attempt == 0) {
+            const float q = (qc == kQUniform) ? q_uniform : sparse_lookup(sid, sval, max(qc, 0), pid[k]);
+            w = __fsub_rn(w, q);
+          }
+          run += fixed_weight(w);
+          if (t < run) {
+            found = k;
+            break;
+          }
+        }
+      }
+      break;
+    }
+    if (found >= 0) {
+      sm.res_tok = pid[found];
+      sm.res_prob = pv[found];
     }
   }
   group_sync<NT, BAR>();
