@@ -179,30 +179,38 @@ __device__ __forceinline__ int tile_elem(int lane, int j) {
   return j < 4 ? lane * 4 + j : 128 + lane * 4 + (j - 4);
 }
 
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
 // Merged logits y of the lane's eight elements of a staged tile, as four packed pairs:
 // d = c - u; g = fma(s, d, u); y = g * inv_T, one rounding per operation.  Multiplying by 1.0f is exact,
-// so the last step is skipped when inv_T == 1.
+// so the last step is skipped when inv_T == 1.  ctile / utile are shared-memory addresses.
 template <int DTYPE>
-__device__ __forceinline__ void tile_y8(const unsigned char* ctile, const unsigned char* utile, bool has_u, bool has_t,
-                                        int lane, uint64_t s2, uint64_t t2, float (&y)[8]) {
+__device__ __forceinline__ void tile_y8(uint32_t ctile, uint32_t utile, bool has_u, bool has_t, int lane, uint64_t s2,
+                                        uint64_t t2, float (&y)[8]) {
   uint64_t c[4], u[4];
   if (DTYPE == 1) {
-    const uint4 w = *reinterpret_cast<const uint4*>(ctile + lane * 16);
+    const uint4 w = lds128(ctile + lane * 16);
     c[0] = pack2(bf16_lo(w.x), bf16_hi(w.x)); c[1] = pack2(bf16_lo(w.y), bf16_hi(w.y));
     c[2] = pack2(bf16_lo(w.z), bf16_hi(w.z)); c[3] = pack2(bf16_lo(w.w), bf16_hi(w.w));
     if (has_u) {
-      const uint4 v = *reinterpret_cast<const uint4*>(utile + lane * 16);
+      const uint4 v = lds128(utile + lane * 16);
       u[0] = pack2(bf16_lo(v.x), bf16_hi(v.x)); u[1] = pack2(bf16_lo(v.y), bf16_hi(v.y));
       u[2] = pack2(bf16_lo(v.z), bf16_hi(v.z)); u[3] = pack2(bf16_lo(v.w), bf16_hi(v.w));
     }
   } else {
-    const float4 a = *reinterpret_cast<const float4*>(ctile + lane * 16);
-    const float4 b = *reinterpret_cast<const float4*>(ctile + 512 + lane * 16);
-    c[0] = pack2(a.x, a.y); c[1] = pack2(a.z, a.w); c[2] = pack2(b.x, b.y); c[3] = pack2(b.z, b.w);
+    const uint4 a = lds128(ctile + lane * 16);
+    const uint4 b = lds128(ctile + 512 + lane * 16);
+    c[0] = (uint64_t)a.x | ((uint64_t)a.y << 32); c[1] = (uint64_t)a.z | ((uint64_t)a.w << 32);
+    c[2] = (uint64_t)b.x | ((uint64_t)b.y << 32); c[3] = (uint64_t)b.z | ((uint64_t)b.w << 32);
     if (has_u) {
-      const float4 p = *reinterpret_cast<const float4*>(utile + lane * 16);
-      const float4 q = *reinterpret_cast<const float4*>(utile + 512 + lane * 16);
-      u[0] = pack2(p.x, p.y); u[1] = pack2(p.z, p.w); u[2] = pack2(q.x, q.y); u[3] = pack2(q.z, q.w);
+      const uint4 p = lds128(utile + lane * 16);
+      const uint4 q = lds128(utile + 512 + lane * 16);
+      u[0] = (uint64_t)p.x | ((uint64_t)p.y << 32); u[1] = (uint64_t)p.z | ((uint64_t)p.w << 32);
+      u[2] = (uint64_t)q.x | ((uint64_t)q.y << 32); u[3] = (uint64_t)q.z | ((uint64_t)q.w << 32);
     }
   }
 #pragma unroll
@@ -274,8 +282,9 @@ __device__ __forceinline__ PipeSmem<NF> carve_pipe_smem(unsigned char* base, int
   static_assert(sizeof(uint32_t) * kSelBins <= sizeof(int32_t) * kKcapMax, "sel must fit under st_ids");
   static_assert(sizeof(Candidate) * kBinListCap <= sizeof(float) * kKcapMax, "binlist must fit under st_vals");
   PipeSmem<NF> s;
-  uintptr_t p = (reinterpret_cast<uintptr_t>(base) + 127) & ~(uintptr_t)127;
-  s.ring = reinterpret_cast<unsigned char*>(p);
+  // plain pointer arithmetic on the shared array, so that the compiler keeps the shared address space
+  unsigned char* p = base + ((128u - (smem_u32(base) & 127u)) & 127u);
+  s.ring = p;
   p += (size_t)n_stages * 2 * kStageArrayBytes;
   s.ylist = reinterpret_cast<uint64_t*>(p);
   p += (size_t)kListCap * NF * 32 * 8;
@@ -424,8 +433,8 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
           // sample tiles are isolated in the row: one copy per tile, spread over the lanes
           for (int j = lane; j < nt; j += 32) {
             const size_t goff = (size_t)(s * TPS + j) * sched.ss * TR::kTileBytes;
-            bulk_g2s(dst_c + (size_t)j * TR::kTileBytes, gc + goff, TR::kTileBytes, &sm.full[slot]);
-            if (has_u) bulk_g2s(dst_u + (size_t)j * TR::kTileBytes, gu + goff, TR::kTileBytes, &sm.full[slot]);
+            bulk_g2s(dst_c + (uint32_t)j * TR::kTileBytes, gc + goff, TR::kTileBytes, &sm.full[slot]);
+            if (has_u) bulk_g2s(dst_u + (uint32_t)j * TR::kTileBytes, gu + goff, TR::kTileBytes, &sm.full[slot]);
           }
         } else {
           // tail tiles come in runs of SS-1 contiguous tiles: lane r copies the r-th run of the stage
@@ -470,6 +479,7 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
     const int fw = warp;
     const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
     const bool has_t = a.inv_T != 1.0f;
+    const uint32_t ring_addr = smem_u32(sm.ring);
     const uint32_t list_base = smem_u32(sm.ylist) + (uint32_t)tid * 8u;
     const uint32_t list_limit = list_base + (uint32_t)(kListCap - 4) * kStride;  // beyond it a tile may not fit
     int slot = 0, flip = 0;
@@ -490,12 +500,12 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
         for (int s = 0; s < sched.sample_stages && ok; ++s) {
           ok = mbar_wait(&sm.full[sl], ph);
           if (ok) {
-            const unsigned char* st_c = sm.ring + (size_t)sl * TR::kStageBytes;
-            const unsigned char* st_u = st_c + kStageArrayBytes;
+            const uint32_t st_c = ring_addr + (uint32_t)sl * TR::kStageBytes;
+            const uint32_t st_u = st_c + kStageArrayBytes;
             const int nt = sched.stage_tiles(s, TPS);
             for (int j = fw; j < nt; j += NF) {
               float y[8];
-              tile_y8<DTYPE>(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes, has_u, has_t, lane, s2,
+              tile_y8<DTYPE>(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes, has_u, has_t, lane, s2,
                              t2, y);
               const float m8 = max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]);
               atomicAdd(&sm.hist[float_key(canonical(m8)) >> 21], 1u);
@@ -530,12 +540,12 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
         // ---------------- sample, pass B: linear bins over [floor, sample max] ----------------
         int sl = slot;
         for (int s = 0; s < sched.sample_stages; ++s) {
-          const unsigned char* st_c = sm.ring + (size_t)sl * TR::kStageBytes;
-          const unsigned char* st_u = st_c + kStageArrayBytes;
+          const uint32_t st_c = ring_addr + (uint32_t)sl * TR::kStageBytes;
+          const uint32_t st_u = st_c + kStageArrayBytes;
           const int nt = sched.stage_tiles(s, TPS);
           for (int j = fw; j < nt; j += NF) {
             float y[8];
-            tile_y8<DTYPE>(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes, has_u, has_t, lane, s2, t2,
+            tile_y8<DTYPE>(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes, has_u, has_t, lane, s2, t2,
                            y);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -574,7 +584,7 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       // One tile: four pairs.  Pair k is stored at cur + k*stride minus one stride for every earlier miss
       // of this tile; z < 0 (sign bit set) marks a miss.  A pair of NaNs counts as a hit and is dropped
       // later; -inf never hits.
-      auto filter_tile = [&](const unsigned char* ctile, const unsigned char* utile) {
+      auto filter_tile = [&](uint32_t ctile, uint32_t utile) {
         float y[8];
         tile_y8<DTYPE>(ctile, utile, has_u, has_t, lane, s2, t2, y);
         if (cur > list_limit) {
@@ -601,10 +611,10 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       };
       // ---------------- the sample tiles, now against tau0 ----------------
       for (int s = 0; s < sched.sample_stages; ++s) {
-        const unsigned char* st_c = sm.ring + (size_t)slot * TR::kStageBytes;
-        const unsigned char* st_u = st_c + kStageArrayBytes;
+        const uint32_t st_c = ring_addr + (uint32_t)slot * TR::kStageBytes;
+        const uint32_t st_u = st_c + kStageArrayBytes;
         const int nt = sched.stage_tiles(s, TPS);
-        for (int j = fw; j < nt; j += NF) filter_tile(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes);
+        for (int j = fw; j < nt; j += NF) filter_tile(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes);
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.empty[slot]);
         if (++slot == NS) {
@@ -616,10 +626,10 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
       for (int s = sched.sample_stages; s < sched.stages; ++s) {
         if (ok) ok = mbar_wait(&sm.full[slot], phase);
         if (ok) {
-          const unsigned char* st_c = sm.ring + (size_t)slot * TR::kStageBytes;
-          const unsigned char* st_u = st_c + kStageArrayBytes;
+          const uint32_t st_c = ring_addr + (uint32_t)slot * TR::kStageBytes;
+          const uint32_t st_u = st_c + kStageArrayBytes;
           const int nt = sched.stage_tiles(s, TPS);
-          for (int j = fw; j < nt; j += NF) filter_tile(st_c + (size_t)j * TR::kTileBytes, st_u + (size_t)j * TR::kTileBytes);
+          for (int j = fw; j < nt; j += NF) filter_tile(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.empty[slot]);
