@@ -37,7 +37,7 @@ constexpr int kTileElems = 256;           // elements per tile: one warp iterati
 constexpr int kStageArrayBytes = 8192;    // bytes of ONE logits array in a ring stage
 constexpr int kHistBins = 2048;           // filter's sample histogram (group maxima by key, then linear bins)
 constexpr int kSelBins = 2048;            // finisher's linear bins over [tau0, max]
-constexpr int kListCap = 32;              // pair entries per filter thread and row (the last four are slack
+constexpr int kListCap = 36;              // pair entries per filter thread and row (the last four are slack
                                           // for the unconditional stores of one tile)
 constexpr int kMaskWordsMax = 8;          // 32 hit bits each: up to 64 tiles per filter warp and row
 constexpr int kItersMax = 64;
@@ -188,9 +188,9 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 // Merged logits y of the lane's eight elements of a staged tile, as four packed pairs:
 // d = c - u; g = fma(s, d, u); y = g * inv_T, one rounding per operation.  Multiplying by 1.0f is exact,
 // so the last step is skipped when inv_T == 1.  ctile / utile are shared-memory addresses.
-template <int DTYPE>
-__device__ __forceinline__ void tile_y8(uint32_t ctile, uint32_t utile, bool has_u, bool has_t, int lane, uint64_t s2,
-                                        uint64_t t2, float (&y)[8]) {
+template <int DTYPE, bool has_u, bool has_t>
+__device__ __forceinline__ void tile_y8(uint32_t ctile, uint32_t utile, int lane, uint64_t s2, uint64_t t2,
+                                        float (&y)[8]) {
   uint64_t c[4], u[4];
   if (DTYPE == 1) {
     const uint4 w = lds128(ctile + lane * 16);
@@ -361,11 +361,200 @@ __device__ __forceinline__ float key_float(uint32_t key) {
   return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
+// The filter warps' loop over this CTA's rows (see the head of the file).  BAR_F = 1 is their named barrier.
+template <int DTYPE, int NF, bool HAS_U, bool HAS_T>
+__device__ __forceinline__ void filter_role(const RowArgs& a, const PipeCfg& cfg, const PipeSmem<NF>& sm,
+                                            const RowSchedule& sched) {
+  constexpr int NT_F = NF * 32;
+  constexpr int BAR_F = 1;
+  constexpr uint32_t kStride = NT_F * 8;  // bytes between consecutive entries of one filter thread
+  using TR = PipeTraits<DTYPE>;
+  constexpr int TPS = TR::kTilesPerStage;
+  const int tid = threadIdx.x, lane = threadIdx.x & 31, fw = threadIdx.x >> 5;
+  const int NS = cfg.n_stages, mask_words = cfg.mask_words;
+  const int rows = a.B * a.W;
+  const float neg_inf = __int_as_float(0xff800000);
+  const float lowest = -3.402823466e38f;  // with this threshold every finite value is a candidate
+  volatile int* abort_flag = sm.ctl + kCtlAbort;
+  const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
+  const uint32_t ring_addr = smem_u32(sm.ring);
+  const uint32_t list_base = smem_u32(sm.ylist) + (uint32_t)tid * 8u;
+  const uint32_t list_limit = list_base + (uint32_t)(kListCap - 4) * kStride;  // beyond it a tile may not fit
+  int slot = 0, flip = 0;
+  uint32_t phase = 0;
+  uint32_t n_row = 0;
+  bool dead = false;
+  for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    const int b = row / a.W, i = row - b * a.W;
+    const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
+    if (i >= L || dead) continue;
+
+    // ---------------- sample, first pass: maxima of groups of eight, by key ----------------
+    bool ok = true;
+    float smax = neg_inf;
+    {
+      int sl = slot;
+      uint32_t ph = phase;
+      for (int s = 0; s < sched.sample_stages && ok; ++s) {
+        ok = mbar_wait(&sm.full[sl], ph);
+        if (ok) {
+          const uint32_t st_c = ring_addr + (uint32_t)sl * TR::kStageBytes;
+          const uint32_t st_u = st_c + kStageArrayBytes;
+          const int nt = sched.stage_tiles(s, TPS);
+          for (int j = fw; j < nt; j += NF) {
+            float y[8];
+            tile_y8<DTYPE, HAS_U, HAS_T>(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes, lane, s2,
+                                         t2, y);
+            const float m8 = max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]);
+            atomicAdd(&sm.hist[float_key(canonical(m8)) >> 21], 1u);
+            smax = fmaxf(smax, m8);
+          }
+        }
+        if (++sl == NS) {
+          sl = 0;
+          ph ^= 1u;
+        }
+      }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, d));
+    if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(&sm.ctl[kCtlSmaxKey]), float_key(canonical(smax)));
+    // lists and hit bits must be back from the finisher before anything is appended
+    if (ok && n_row > 0) ok = mbar_wait(sm.cand_free, (n_row - 1) & 1u);
+    dead = group_any<NT_F, BAR_F>(!ok);
+    if (dead) {
+      if (tid == 0) *abort_flag = 1;
+      continue;
+    }
+    // at least m group maxima, hence at least m sample elements, are >= the lower edge of this bin
+    find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kCtlFBin);
+    const int cbin = sm.ctl[kCtlFBin];
+    float floor_y = cbin >= 0 ? key_float((uint32_t)cbin << 21) : lowest;
+    if (!(floor_y >= lowest)) floor_y = lowest;  // edge fell on -inf or into the NaN patterns
+    const float top_y = key_float((uint32_t)sm.ctl[kCtlSmaxKey]);
+    const bool refine = floor_y > lowest && top_y >= floor_y && top_y <= 3.402823466e38f;
+    const float range = __fsub_rn(top_y, floor_y);
+    const float scale = (refine && range > 0.0f) ? __fdiv_rn((float)kHistBins - 0.5f, range) : 0.0f;
+
+    uint32_t cur = list_base;  // shared-memory address of the thread's next free entry
+    uint32_t imw = 0;          // inverted hit bits of the last (it & 7) tiles
+    int it = 0;                // tiles this warp has filtered in this row
+    bool overflow = false;
+    // One tile: four pairs.  A pair is always stored at the cursor; the cursor moves on only for a hit,
+    // i.e. when max(pair) - thr has no sign bit.  A pair of NaNs counts as a hit and is dropped later; -inf
+    // never hits.
+    auto filter_tile = [&](uint32_t ctile, uint32_t utile, float thr) {
+      float y[8];
+      tile_y8<DTYPE, HAS_U, HAS_T>(ctile, utile, lane, s2, t2, y);
+      if (cur > list_limit) {
+        overflow = true;
+        cur = list_base;
+      }
+      uint32_t d = cur;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float m = fmaxf(y[2 * k], y[2 * k + 1]);
+        const uint32_t miss = __umulhi(__float_as_uint(__fsub_rn(m, thr)), 2u);
+        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(d), "f"(y[2 * k]), "f"(y[2 * k + 1]) : "memory");
+        d = d + kStride - miss * kStride;
+        imw = imw * 2u + miss;
+      }
+      cur = d;
+      ++it;
+      if ((it & 7) == 0) {
+        if ((it >> 3) <= mask_words) sm.masks[(size_t)((it >> 3) - 1) * NT_F + tid] = imw;
+        imw = 0;
+      }
+    };
+    // ---------------- the sample tiles against the floor (a superset of what tau0 will keep) ----------------
+    const float sample_thr = refine ? floor_y : lowest;
+    for (int s = 0; s < sched.sample_stages; ++s) {
+      const uint32_t st_c = ring_addr + (uint32_t)slot * TR::kStageBytes;
+      const uint32_t st_u = st_c + kStageArrayBytes;
+      const int nt = sched.stage_tiles(s, TPS);
+      for (int j = fw; j < nt; j += NF)
+        filter_tile(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes, sample_thr);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.empty[slot]);
+      if (++slot == NS) {
+        slot = 0;
+        phase ^= 1u;
+      }
+    }
+    // ---------------- sample, second pass: linear bins over [floor, sample max], from the lists ----------------
+    float tau0 = lowest;
+    if (refine) {
+      for (uint32_t e = list_base; e < cur; e += kStride) {
+        float v0, v1;
+        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v0), "=f"(v1) : "r"(e));
+        if (v0 >= floor_y) {
+          const int q = __float2int_rd(__fmul_rn(__fsub_rn(v0, floor_y), scale));
+          atomicAdd(&sm.hist[min(max(q, 0), kHistBins - 1)], 1u);
+        }
+        if (v1 >= floor_y) {
+          const int q = __float2int_rd(__fmul_rn(__fsub_rn(v1, floor_y), scale));
+          atomicAdd(&sm.hist[min(max(q, 0), kHistBins - 1)], 1u);
+        }
+      }
+      group_sync<NT_F, BAR_F>();
+      if (tid == 0) sm.ctl[kCtlSmaxKey] = 0;  // every thread has read it; next written after the next row's barriers
+      find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kCtlFBin);
+      const int fbin = sm.ctl[kCtlFBin];
+      if (fbin > 0 && scale > 0.0f) {
+        // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
+        const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
+        tau0 = __fadd_rd(floor_y, t);
+      } else if (fbin >= 0) {
+        tau0 = floor_y;
+      }
+    } else {
+      group_sync<NT_F, BAR_F>();
+      if (tid == 0) sm.ctl[kCtlSmaxKey] = 0;
+    }
+    // ---------------- the rest of the row against tau0 ----------------
+    for (int s = sched.sample_stages; s < sched.stages; ++s) {
+      if (ok) ok = mbar_wait(&sm.full[slot], phase);
+      if (ok) {
+        const uint32_t st_c = ring_addr + (uint32_t)slot * TR::kStageBytes;
+        const uint32_t st_u = st_c + kStageArrayBytes;
+        const int nt = sched.stage_tiles(s, TPS);
+        for (int j = fw; j < nt; j += NF)
+          filter_tile(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes, tau0);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.empty[slot]);
+      if (++slot == NS) {
+        slot = 0;
+        phase ^= 1u;
+      }
+    }
+    // ---------------- hand the row over ----------------
+    {
+      const int rem = it & 7;
+      int w = it >> 3;
+      if (rem != 0 && w < mask_words) {
+        const int fill = 32 - 4 * rem;  // bits of the word not reached: misses
+        sm.masks[(size_t)w * NT_F + tid] = (imw << fill) | ((1u << fill) - 1u);
+        ++w;
+      }
+      for (; w < mask_words; ++w) sm.masks[(size_t)w * NT_F + tid] = 0xffffffffu;
+      if (overflow) sm.ctl[kCtlRowOverflow] = 1;
+      if (tid == 0) sm.ctl[kCtlRowTau0] = __float_as_int(tau0);
+    }
+    dead = group_any<NT_F, BAR_F>(!ok);
+    if (dead) {
+      if (tid == 0) *abort_flag = 1;
+      continue;  // the row is not handed over: the finisher's wait runs out and marks the rows
+    }
+    if (lane == 0) mbar_arrive(sm.cand_full);
+    ++n_row;
+  }
+}
+
 template <int DTYPE, int NF, int NP>
 __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(const RowArgs a, const PipeCfg cfg) {
   constexpr int NT_F = NF * 32, NT_P = NP * 32;
   constexpr int BAR_F = 1, BAR_P = 2;
-  constexpr uint32_t kStride = NT_F * 8;  // bytes between consecutive entries of one filter thread
   static_assert(NF <= 16 && NP * 32 * kFinItems >= kKcapMax, "group sizes");
   using TR = PipeTraits<DTYPE>;
   constexpr int TPS = TR::kTilesPerStage;
@@ -475,189 +664,13 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
 
   if (warp < NF) {
     // ======================================= filter warps =======================================
-    const int tid = threadIdx.x;  // 0 .. NT_F-1
-    const int fw = warp;
-    const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
     const bool has_t = a.inv_T != 1.0f;
-    const uint32_t ring_addr = smem_u32(sm.ring);
-    const uint32_t list_base = smem_u32(sm.ylist) + (uint32_t)tid * 8u;
-    const uint32_t list_limit = list_base + (uint32_t)(kListCap - 4) * kStride;  // beyond it a tile may not fit
-    int slot = 0, flip = 0;
-    uint32_t phase = 0;
-    uint32_t n_row = 0;
-    bool dead = false;
-    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-      const int b = row / a.W, i = row - b * a.W;
-      const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
-      if (i >= L || dead) continue;
-
-      // ---------------- sample, pass A: maxima of groups of eight, by key ----------------
-      bool ok = true;
-      float smax = neg_inf;
-      {
-        int sl = slot;
-        uint32_t ph = phase;
-        for (int s = 0; s < sched.sample_stages && ok; ++s) {
-          ok = mbar_wait(&sm.full[sl], ph);
-          if (ok) {
-            const uint32_t st_c = ring_addr + (uint32_t)sl * TR::kStageBytes;
-            const uint32_t st_u = st_c + kStageArrayBytes;
-            const int nt = sched.stage_tiles(s, TPS);
-            for (int j = fw; j < nt; j += NF) {
-              float y[8];
-              tile_y8<DTYPE>(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes, has_u, has_t, lane, s2,
-                             t2, y);
-              const float m8 = max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]);
-              atomicAdd(&sm.hist[float_key(canonical(m8)) >> 21], 1u);
-              smax = fmaxf(smax, m8);
-            }
-          }
-          if (++sl == NS) {
-            sl = 0;
-            ph ^= 1u;
-          }
-        }
-      }
-#pragma unroll
-      for (int d = 16; d > 0; d >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, d));
-      if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(&sm.ctl[kCtlSmaxKey]), float_key(canonical(smax)));
-      dead = group_any<NT_F, BAR_F>(!ok);
-      if (dead) {
-        if (tid == 0) *abort_flag = 1;
-        continue;
-      }
-      // at least m group maxima, hence at least m sample elements, are >= the lower edge of this bin
-      find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kCtlFBin);
-      const int cbin = sm.ctl[kCtlFBin];
-      float floor_y = cbin >= 0 ? key_float((uint32_t)cbin << 21) : lowest;
-      if (!(floor_y >= lowest)) floor_y = lowest;  // edge fell on -inf or into the NaN patterns
-      const float top_y = key_float((uint32_t)sm.ctl[kCtlSmaxKey]);
-      const bool refine = floor_y > lowest && top_y >= floor_y && top_y <= 3.402823466e38f;
-      const float range = __fsub_rn(top_y, floor_y);
-      const float scale = (refine && range > 0.0f) ? __fdiv_rn((float)kHistBins - 0.5f, range) : 0.0f;
-      float tau0 = lowest;
-      if (refine) {
-        // ---------------- sample, pass B: linear bins over [floor, sample max] ----------------
-        int sl = slot;
-        for (int s = 0; s < sched.sample_stages; ++s) {
-          const uint32_t st_c = ring_addr + (uint32_t)sl * TR::kStageBytes;
-          const uint32_t st_u = st_c + kStageArrayBytes;
-          const int nt = sched.stage_tiles(s, TPS);
-          for (int j = fw; j < nt; j += NF) {
-            float y[8];
-            tile_y8<DTYPE>(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes, has_u, has_t, lane, s2, t2,
-                           y);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              if (y[e] >= floor_y) {
-                const int q = __float2int_rd(__fmul_rn(__fsub_rn(y[e], floor_y), scale));
-                atomicAdd(&sm.hist[min(max(q, 0), kHistBins - 1)], 1u);
-              }
-            }
-          }
-          if (++sl == NS) sl = 0;
-        }
-        group_sync<NT_F, BAR_F>();
-        find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kCtlFBin);
-        const int fbin = sm.ctl[kCtlFBin];
-        if (fbin > 0 && scale > 0.0f) {
-          // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
-          const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
-          tau0 = __fadd_rd(floor_y, t);
-        } else if (fbin == 0 || (fbin > 0 && scale == 0.0f)) {
-          tau0 = floor_y;
-        }
-      }
-      // ---------------- lists and hit bits must be back from the finisher ----------------
-      if (n_row > 0) ok = mbar_wait(sm.cand_free, (n_row - 1) & 1u);
-      dead = group_any<NT_F, BAR_F>(!ok);
-      if (dead) {
-        if (tid == 0) *abort_flag = 1;
-        continue;
-      }
-      if (tid == 0) sm.ctl[kCtlSmaxKey] = 0;  // every thread has read it; next written after the next row's barriers
-
-      uint32_t cur = list_base;  // shared-memory address of the thread's next free entry
-      uint32_t imw = 0;          // inverted hit bits of the last (it & 7) tiles
-      int it = 0;                // tiles this warp has filtered in this row
-      bool overflow = false;
-      // One tile: four pairs.  Pair k is stored at cur + k*stride minus one stride for every earlier miss
-      // of this tile; z < 0 (sign bit set) marks a miss.  A pair of NaNs counts as a hit and is dropped
-      // later; -inf never hits.
-      auto filter_tile = [&](uint32_t ctile, uint32_t utile) {
-        float y[8];
-        tile_y8<DTYPE>(ctile, utile, has_u, has_t, lane, s2, t2, y);
-        if (cur > list_limit) {
-          overflow = true;
-          cur = list_base;
-        }
-        uint32_t d = cur;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float m = fmaxf(y[2 * k], y[2 * k + 1]);
-          const uint32_t miss = __umulhi(__float_as_uint(__fsub_rn(m, tau0)), 2u);
-          asm volatile("st.shared.v2.f32 [%0+%3], {%1, %2};" ::"r"(d), "f"(y[2 * k]), "f"(y[2 * k + 1]),
-                       "n"(0)
-                       : "memory");
-          d = d + kStride - miss * kStride;
-          imw = imw * 2u + miss;
-        }
-        cur = d;
-        ++it;
-        if ((it & 7) == 0) {
-          if ((it >> 3) <= mask_words) sm.masks[(size_t)((it >> 3) - 1) * NT_F + tid] = imw;
-          imw = 0;
-        }
-      };
-      // ---------------- the sample tiles, now against tau0 ----------------
-      for (int s = 0; s < sched.sample_stages; ++s) {
-        const uint32_t st_c = ring_addr + (uint32_t)slot * TR::kStageBytes;
-        const uint32_t st_u = st_c + kStageArrayBytes;
-        const int nt = sched.stage_tiles(s, TPS);
-        for (int j = fw; j < nt; j += NF) filter_tile(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.empty[slot]);
-        if (++slot == NS) {
-          slot = 0;
-          phase ^= 1u;
-        }
-      }
-      // ---------------- the rest of the row ----------------
-      for (int s = sched.sample_stages; s < sched.stages; ++s) {
-        if (ok) ok = mbar_wait(&sm.full[slot], phase);
-        if (ok) {
-          const uint32_t st_c = ring_addr + (uint32_t)slot * TR::kStageBytes;
-          const uint32_t st_u = st_c + kStageArrayBytes;
-          const int nt = sched.stage_tiles(s, TPS);
-          for (int j = fw; j < nt; j += NF) filter_tile(st_c + (uint32_t)j * TR::kTileBytes, st_u + (uint32_t)j * TR::kTileBytes);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.empty[slot]);
-        if (++slot == NS) {
-          slot = 0;
-          phase ^= 1u;
-        }
-      }
-      // ---------------- hand the row over ----------------
-      {
-        const int rem = it & 7;
-        int w = it >> 3;
-        if (rem != 0 && w < mask_words) {
-          const int fill = 32 - 4 * rem;  // bits of the word not reached: misses
-          sm.masks[(size_t)w * NT_F + tid] = (imw << fill) | ((1u << fill) - 1u);
-          ++w;
-        }
-        for (; w < mask_words; ++w) sm.masks[(size_t)w * NT_F + tid] = 0xffffffffu;
-        if (overflow) sm.ctl[kCtlRowOverflow] = 1;
-        if (tid == 0) sm.ctl[kCtlRowTau0] = __float_as_int(tau0);
-      }
-      dead = group_any<NT_F, BAR_F>(!ok);
-      if (dead) {
-        if (tid == 0) *abort_flag = 1;
-        continue;  // the row is not handed over: the finisher's wait runs out and marks the rows
-      }
-      if (lane == 0) mbar_arrive(sm.cand_full);
-      ++n_row;
+    if (has_u) {
+      if (has_t) filter_role<DTYPE, NF, true, true>(a, cfg, sm, sched);
+      else filter_role<DTYPE, NF, true, false>(a, cfg, sm, sched);
+    } else {
+      if (has_t) filter_role<DTYPE, NF, false, true>(a, cfg, sm, sched);
+      else filter_role<DTYPE, NF, false, false>(a, cfg, sm, sched);
     }
     return;
   }

@@ -83,8 +83,9 @@ bool plan_pipeline(const sjd_params* P, int kcap, sjd::PipeCfg* cfg, size_t* sme
     if (m > n_sample / 2 || m > 32 * sample_tiles) continue;  // the rank must exist among the group maxima too
     const double mean = (double)m * ss, sd = (double)ss * std::sqrt((double)m);
     if (mean + 4.0 * sd > (double)sjd::kDenseCap) continue;
-    const double per_thread = mean / (32.0 * kFilterWarps);
-    if (per_thread + 5.5 * std::sqrt(per_thread) + 1.0 > (double)(sjd::kListCap - 4)) continue;
+    // sample pairs are kept against a floor somewhat below the threshold: about 2m more entries
+    const double per_thread = (mean + 2.0 * m) / (32.0 * kFilterWarps);
+    if (per_thread + 5.0 * std::sqrt(per_thread) + 1.0 > (double)(sjd::kListCap - 4)) continue;
     cfg->sample_stride = ss;
     cfg->sample_rank = m;
     cfg->n_stages = ns;
