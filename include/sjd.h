@@ -161,6 +161,36 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
              int32_t* out_accept_len, int32_t* out_tokens, sjd_probs* out_probs);
 
 /*
+ * Window bookkeeping of the decode loop (Section 4.1: Step 1 "draft token preparation", the last sentence
+ * of Step 3 "accepted tokens are appended", the last sentence of Step 4 "accepted and reinitialised tokens
+ * form the next window"; random initialisation is the baseline of Section 4.2).
+ *
+ * sjd_window_init() fills the first window: drafts[b,i] for i < win_len[b] is a token drawn uniformly from
+ * [0,V) (Philox purpose 4, counter = (pos_base[b]+i, seq_base+b, iteration[b], 4), token = floor(x0 V / 2^32))
+ * and its reference distribution is SJD_Q_UNIFORM with tok_prob = 1/V; rows beyond win_len get token -1.
+ *
+ * sjd_window_advance() takes what sjd_step() just produced (accept_len, out_tokens, out_probs) and
+ *   - commits c_b tokens per sequence: the accepted prefix plus the residual draw at the first rejected row
+ *     (c = a+1), or the whole window when every row was accepted (c = win_len); they are written to
+ *     committed[b, pos_base[b] .. pos_base[b]+c) (committed is [B, n_total] device int32) and c to
+ *     n_committed[b] when that is not NULL;
+ *   - builds the next window in next_drafts / next_probs (which must not alias the step's outputs): row i takes
+ *     the step's row i+c with that row's distribution as its reference when i+c < win_len, else a newly
+ *     initialised token as in sjd_window_init() with the iteration index of the step that just ran;
+ *   - updates win_len, pos_base, iteration in place: pos_base += c, win_len = min(W, n_total - pos_base),
+ *     iteration += 1.  A sequence is finished when its win_len is 0.
+ * params supplies B, W, V, top_k, seq_base and stream; its win_len/pos_base/iteration fields are not used
+ * (the arrays are passed explicitly because they are written).  All pointers are device pointers.  Both
+ * calls are asynchronous on params->stream and return SJD_OK or a negative SJD_ERR_*.
+ */
+int sjd_window_init(const sjd_params* params, int32_t n_total, uint64_t philox_seed, int32_t* win_len, int32_t* pos_base,
+                    int32_t* iteration, int32_t* drafts, sjd_probs* draft_probs);
+int sjd_window_advance(const sjd_params* params, int32_t n_total, uint64_t philox_seed, const int32_t* accept_len,
+                       const int32_t* step_tokens, const sjd_probs* step_probs, int32_t* win_len, int32_t* pos_base,
+                       int32_t* iteration, int32_t* next_drafts, sjd_probs* next_probs, int32_t* committed,
+                       int32_t* n_committed);
+
+/*
  * sjd_step() for callers that cannot hand over a workspace.  (The paper has no counterpart: this is a
  * convenience of this library, not a step of the method.)
  *

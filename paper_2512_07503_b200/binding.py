@@ -62,6 +62,13 @@ def lib() -> C.CDLL:
         L.sjd_step.restype = C.c_int
         L.sjd_step_static.argtypes = L.sjd_step.argtypes
         L.sjd_step_static.restype = C.c_int
+        L.sjd_window_init.argtypes = [C.POINTER(sjd_params), C.c_int32, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.POINTER(sjd_probs)]
+        L.sjd_window_init.restype = C.c_int
+        L.sjd_window_advance.argtypes = [C.POINTER(sjd_params), C.c_int32, C.c_uint64, C.c_void_p, C.c_void_p,
+                                         C.POINTER(sjd_probs), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.POINTER(sjd_probs), C.c_void_p, C.c_void_p]
+        L.sjd_window_advance.restype = C.c_int
         _lib = L
     return _lib
 
@@ -186,6 +193,32 @@ def sjd_step(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor], d
                               _opt_ptr(drafts), C.byref(q) if q is not None else None, C.byref(params),
                               int(philox_seed) & 0xFFFFFFFFFFFFFFFF, _opt_ptr(out_accept_len), _opt_ptr(out_tokens),
                               C.byref(o))
+    _check(code)
+
+
+def sjd_window_init(params: sjd_params, n_total: int, philox_seed: int, win_len: torch.Tensor, pos_base: torch.Tensor,
+                    iteration: torch.Tensor, drafts: torch.Tensor, draft_probs: DeviceProbs) -> None:
+    """Fill the first window with randomly initialised drafts (uniform reference distribution)."""
+    q = draft_probs.c_struct()
+    with torch.cuda.device(drafts.device):
+        code = lib().sjd_window_init(C.byref(params), int(n_total), int(philox_seed) & 0xFFFFFFFFFFFFFFFF,
+                                     _opt_ptr(win_len), _opt_ptr(pos_base), _opt_ptr(iteration), _opt_ptr(drafts),
+                                     C.byref(q))
+    _check(code)
+
+
+def sjd_window_advance(params: sjd_params, n_total: int, philox_seed: int, accept_len: torch.Tensor,
+                       step_tokens: torch.Tensor, step_probs: DeviceProbs, win_len: torch.Tensor, pos_base: torch.Tensor,
+                       iteration: torch.Tensor, next_drafts: torch.Tensor, next_probs: DeviceProbs,
+                       committed: torch.Tensor, n_committed: Optional[torch.Tensor] = None) -> None:
+    """Commit the accepted prefix and the residual token, shift the window and refill it (same arguments as
+    the C entry point)."""
+    sp, nq = step_probs.c_struct(), next_probs.c_struct()
+    with torch.cuda.device(step_tokens.device):
+        code = lib().sjd_window_advance(C.byref(params), int(n_total), int(philox_seed) & 0xFFFFFFFFFFFFFFFF,
+                                        _opt_ptr(accept_len), _opt_ptr(step_tokens), C.byref(sp), _opt_ptr(win_len),
+                                        _opt_ptr(pos_base), _opt_ptr(iteration), _opt_ptr(next_drafts), C.byref(nq),
+                                        _opt_ptr(committed), _opt_ptr(n_committed))
     _check(code)
 
 

@@ -13,6 +13,7 @@
 #include "row_kernels.cuh"
 #include "rows_pipeline.cuh"
 #include "verify_kernel.cuh"
+#include "advance_kernel.cuh"
 
 #include <cmath>
 
@@ -298,6 +299,73 @@ int sjd_step_static(const void* logits_cond, const void* logits_uncond, const in
   Q.workspace = scratch;
   Q.workspace_bytes = kStaticScratchBytes;
   return sjd_step(logits_cond, logits_uncond, drafts, draft_probs, &Q, philox_seed, out_accept_len, out_tokens, out_probs);
+}
+
+}  // extern "C"
+
+namespace {
+int fill_advance(sjd::AdvanceArgs* a, const sjd_params* P, int32_t n_total, uint64_t seed, int32_t* win_len,
+                 int32_t* pos_base, int32_t* iteration, int32_t* next_drafts, sjd_probs* next_probs) {
+  if (!P) return SJD_ERR_NULL;
+  if (P->struct_size != (int32_t)sizeof(sjd_params)) return SJD_ERR_STRUCT;
+  if (!win_len || !pos_base || !iteration || !next_drafts || check_probs(next_probs) != SJD_OK) return SJD_ERR_NULL;
+  if (P->B < 0 || P->W < 1 || P->W > SJD_W_MAX || P->V < 1 || P->top_k < 1 || n_total < 0) return SJD_ERR_SHAPE;
+  std::memset(a, 0, sizeof(*a));
+  a->B = P->B; a->W = P->W; a->V = P->V;
+  a->kcap = P->top_k < P->V ? P->top_k : P->V;
+  a->n_total = n_total;
+  a->seq_base = P->seq_base;
+  a->seed_lo = (uint32_t)(seed & 0xffffffffu);
+  a->seed_hi = (uint32_t)(seed >> 32);
+  a->win_len = win_len; a->pos_base = pos_base; a->iteration = iteration;
+  a->next_drafts = next_drafts;
+  a->next_tok_prob = next_probs->tok_prob; a->next_ids = next_probs->ids; a->next_vals = next_probs->vals;
+  a->next_cnt = next_probs->cnt;
+  return SJD_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int sjd_window_init(const sjd_params* P, int32_t n_total, uint64_t philox_seed, int32_t* win_len, int32_t* pos_base,
+                    int32_t* iteration, int32_t* drafts, sjd_probs* draft_probs) {
+  sjd::AdvanceArgs a;
+  const int rc = fill_advance(&a, P, n_total, philox_seed, win_len, pos_base, iteration, drafts, draft_probs);
+  if (rc != SJD_OK) return rc;
+  if (P->B == 0) return SJD_OK;
+  const int rows = P->B * P->W;
+  sjd::init_window_kernel<<<(rows + 255) / 256, 256, 0, static_cast<cudaStream_t>(P->stream)>>>(a);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "window init launch");
+  ++g_launches;
+  return SJD_OK;
+}
+
+int sjd_window_advance(const sjd_params* P, int32_t n_total, uint64_t philox_seed, const int32_t* accept_len,
+                       const int32_t* step_tokens, const sjd_probs* step_probs, int32_t* win_len, int32_t* pos_base,
+                       int32_t* iteration, int32_t* next_drafts, sjd_probs* next_probs, int32_t* committed,
+                       int32_t* n_committed) {
+  sjd::AdvanceArgs a;
+  const int rc = fill_advance(&a, P, n_total, philox_seed, win_len, pos_base, iteration, next_drafts, next_probs);
+  if (rc != SJD_OK) return rc;
+  if (!accept_len || !step_tokens || !committed || check_probs(const_cast<sjd_probs*>(step_probs)) != SJD_OK) return SJD_ERR_NULL;
+  if (P->B == 0) return SJD_OK;
+  a.accept_len = accept_len;
+  a.step_tokens = step_tokens;
+  a.step_tok_prob = step_probs->tok_prob; a.step_ids = step_probs->ids; a.step_vals = step_probs->vals;
+  a.step_cnt = step_probs->cnt;
+  a.committed = committed;
+  a.n_committed = n_committed;
+  cudaStream_t st = static_cast<cudaStream_t>(P->stream);
+  sjd::advance_rows_kernel<256><<<P->B * P->W, 256, 0, st>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "window advance launch");
+  ++g_launches;
+  sjd::advance_state_kernel<<<(P->B + 127) / 128, 128, 0, st>>>(a);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "window state launch");
+  ++g_launches;
+  return SJD_OK;
 }
 
 }  // extern "C"

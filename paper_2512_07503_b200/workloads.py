@@ -139,3 +139,32 @@ def markov_noise(V: int, pos: int, seed: int) -> np.ndarray:
     same logits in every Jacobi iteration."""
     rng = np.random.Generator(np.random.Philox(key=[seed, pos]))
     return rng.standard_normal(V, dtype=np.float32)
+
+
+class MarkovSource:
+    """Synthetic first-order Markov "model" of the decode-loop workload, on the host:
+    cond[pos] = table[prev_token mod states] + noise(seed_c, pos), uncond = cond + noise(seed_u, pos), where
+    prev_token of window row i is the window's own draft at i-1 (the last committed token for row 0, token 0 at
+    the very start), so that a rejection invalidates the later rows' logits.  The noise depends on the position
+    only: an unchanged prefix reproduces the same logits in every iteration.  No method arithmetic here."""
+
+    def __init__(self, V: int, n_total: int, dtype: int, states: int = 1024, sigma: float = 3.0, seed_table: int = 7,
+                 seed_c: int = 5, seed_u: int = 6):
+        self.V, self.N, self.dtype, self.states = V, n_total, dtype, states
+        self.table = markov_table(V, states, sigma, seed_table)
+        self.noise_c = np.stack([markov_noise(V, p, seed_c) for p in range(n_total)])
+        self.noise_u = np.stack([markov_noise(V, p, seed_u) for p in range(n_total)])
+
+    def logits(self, drafts: np.ndarray, win_len: np.ndarray, pos_base: np.ndarray, committed: np.ndarray):
+        """cond, uncond of shape [B,W,V] in the storage type, for the given window state."""
+        B, W = drafts.shape
+        cond = np.zeros((B, W, self.V), np.float32)
+        unc = np.zeros((B, W, self.V), np.float32)
+        for b in range(B):
+            p0 = int(pos_base[b])
+            for i in range(int(win_len[b])):
+                prev = int(drafts[b, i - 1]) if i > 0 else (int(committed[b, p0 - 1]) if p0 > 0 else 0)
+                c = self.table[prev % self.states] + self.noise_c[p0 + i]
+                cond[b, i] = c
+                unc[b, i] = c + self.noise_u[p0 + i]
+        return _store(cond, self.dtype), _store(unc, self.dtype)

@@ -1,0 +1,51 @@
+"""Decode loop on the GPU (sjd_step + sjd_window_advance through the C ABI) in lock-step with the oracle's
+loop on the same synthetic Markov logit source: same committed tokens, same number of iterations, same
+tokens committed per iteration."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import loop
+from paper_2512_07503_b200 import workloads as wk
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64):
+    from paper_2512_07503_b200.decode import DecodeLoop
+    src = wk.MarkovSource(V, N, dtype, states=states)
+    flags = oracle.FLAG_REUSE if reuse else 0
+    ref_committed, ref_steps, ref_counts = loop.decode(
+        lambda w: src.logits(w.drafts, w.win_len, w.pos_base, w.committed), B=B, W=W, V=V, n_total=N, dtype=dtype,
+        top_k=top_k, cfg_scale=3.0, flags=flags, seed=seed, n_threads=8)
+
+    tdt = torch.bfloat16 if dtype == wk.BF16 else torch.float32
+    dl = DecodeLoop(batch=B, window=W, vocab=V, n_total=N, logits_dtype=tdt, top_k=top_k, cfg_scale=3.0, reuse=reuse,
+                    seed=seed, device=DEV)
+
+    def up(a):
+        if dtype == wk.BF16:
+            return torch.from_numpy(a.view(np.int16)).to(DEV).view(torch.bfloat16)
+        return torch.from_numpy(a).to(DEV)
+
+    def source(d):
+        c, u = src.logits(d.window_tokens.cpu().numpy(), d.win_len.cpu().numpy(), d.pos_base.cpu().numpy(),
+                          d.committed.cpu().numpy())
+        return up(c), up(u)
+
+    committed, steps, counts = dl.run(source, max_steps=4 * N)
+    assert int(dl.status.max().item()) & 8 == 0
+    return (committed.numpy(), steps, counts.numpy()), (ref_committed, ref_steps, ref_counts)
+
+
+@pytest.mark.parametrize("B,W,V,N,K,dtype,reuse", [(3, 8, 4096, 50, 64, wk.F32, True), (2, 16, 8192, 70, 300, wk.BF16, True),
+                                                   (2, 5, 512, 23, 40, wk.F32, False), (1, 32, 16384, 96, 1000, wk.BF16, True)])
+def test_loop_matches_the_oracle(B, W, V, N, K, dtype, reuse):
+    got, ref = _both(B, W, V, N, K, dtype, reuse)
+    assert got[1] == ref[1], (got[1], ref[1])
+    assert np.array_equal(got[2], ref[2])
+    assert np.array_equal(got[0], ref[0])
+    assert np.all(got[2].sum(axis=0) == N)
+    print("steps", got[1], "tokens per step", N * B / max(1, got[2].shape[0] * B))
