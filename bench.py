@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--loop", action="store_true",
+                    help="run the full decode loop of the 48x48 grid workload (cfg5) instead of the single-step benchmark")
     return ap.parse_args()
 
 
@@ -423,9 +425,64 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_loop(args):
+    """Decode loop workload: one 48x48 = 2,304-token grid, V=65,536, W=32, bf16, CFG 3.0, top-K 2000, logits
+    from a synthetic first-order Markov source on the device (table row of the previous token + per-position
+    noise).  Reports iterations, mean committed tokens per iteration and the time spent in the library."""
+    import torch
+    import paper_2512_07503_b200 as sjd
+    from paper_2512_07503_b200.decode import DecodeLoop
+    dev = torch.device("cuda", 0)
+    V, N, W, K, states = 65536, 2304, 32, 2000, 1024
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    table = torch.randn(states, V, generator=g, device=dev) * 3.0
+    g.manual_seed(5)
+    noise_c = torch.randn(N, V, generator=g, device=dev).to(torch.bfloat16)
+    g.manual_seed(6)
+    noise_u = torch.randn(N, V, generator=g, device=dev).to(torch.bfloat16)
+    dl = DecodeLoop(batch=1, window=W, vocab=V, n_total=N, logits_dtype=torch.bfloat16, top_k=K, cfg_scale=3.0, seed=5,
+                    device=dev)
+    ar = torch.arange(W, device=dev)
+
+    def source(d):
+        p0 = int(d.pos_base[0].item())
+        L = int(d.win_len[0].item())
+        toks = d.window_tokens[0].long()
+        first = d.committed[0, p0 - 1].long().clamp(min=0) if p0 > 0 else torch.zeros((), dtype=torch.long, device=dev)
+        prev = torch.cat([first.view(1), toks[:W - 1].clamp(min=0)])
+        pos = (p0 + ar).clamp(max=N - 1)
+        cond = table[prev % states] + noise_c[pos].float()
+        cond_s = cond.to(torch.bfloat16)
+        unc_s = (cond_s.float() + noise_u[pos].float()).to(torch.bfloat16)
+        return cond_s.view(1, W, V), unc_s.view(1, W, V)
+
+    ev = []
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    lib_ms = 0.0
+    while not dl.done():
+        cond, unc = source(dl)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        dl.step(cond, unc)
+        b.record()
+        ev.append((a, b))
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    lib_ms = sum(a.elapsed_time(b) for a, b in ev)
+    print(json.dumps({"workload": "cfg5: decode loop, 2304 tokens, V=65536, W=32, bf16, CFG 3.0, top-K 2000, Markov source",
+                      "steps": dl.steps, "tokens": N, "mean_committed_per_step": round(N / dl.steps, 4),
+                      "step_compression_S": round(N / dl.steps, 4), "library_ms_total": round(lib_ms, 3),
+                      "library_us_per_step": round(1e3 * lib_ms / dl.steps, 2), "wall_s_including_logit_source": round(wall, 3),
+                      "complete": bool((dl.committed >= 0).all().item())}), flush=True)
+
+
 if __name__ == "__main__":
     a = parse_args()
-    if a.impl == "reference":
+    if a.loop:
+        run_loop(a)
+    elif a.impl == "reference":
         run_reference(a)
     else:
         run_ours(a)
