@@ -161,7 +161,8 @@ __device__ void row_generic(const RowArgs& a, int row, int tid, GenericSmem& sm)
   group_sync<NT, BAR>();
 
   // ---- softmax over the survivors ----
-  const bool degenerate = (m == __int_as_float(0xff800000));
+  // no finite maximum (nothing finite in the row, or an infinite logit): all probabilities are reported as 0
+  const bool degenerate = !(fabsf(m) <= 3.402823466e38f);
   float zpart = 0.0f;
   for (int k = tid; k < kcap; k += NT) {
     const float e = degenerate ? 0.0f : exp_diff(vals[k], m);

@@ -554,7 +554,7 @@ __device__ __forceinline__ void filter_role(const RowArgs& a, const PipeCfg& cfg
 template <int DTYPE, int NF, int NP>
 __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(const RowArgs a, const PipeCfg cfg) {
   constexpr int NT_F = NF * 32, NT_P = NP * 32;
-  constexpr int BAR_F = 1, BAR_P = 2;
+  constexpr int BAR_P = 2;  // named barrier of the finisher warps (the filter warps use 1)
   static_assert(NF <= 16 && NP * 32 * kFinItems >= kKcapMax, "group sizes");
   using TR = PipeTraits<DTYPE>;
   constexpr int TPS = TR::kTilesPerStage;
@@ -564,7 +564,6 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
   const int NS = cfg.n_stages;
   const bool has_u = a.uncond != nullptr;
   const float neg_inf = __int_as_float(0xff800000);
-  const float lowest = -3.402823466e38f;  // with this threshold every finite value is a candidate
 
   const RowSchedule sched(a.V, cfg.sample_stride, TPS);
   const int rows = a.B * a.W;

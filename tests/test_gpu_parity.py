@@ -140,3 +140,70 @@ def test_bad_arguments_are_refused_on_the_host():
         with pytest.raises(sjd.SjdError, match=f"sjd error {code}"):
             sjd.sjd_step(logits, None, None, None, p, 0, acc, toks, out)
     torch.cuda.synchronize()
+
+
+# ---- shapes the single-pass pipelined kernel takes, driven into its rare paths ----
+def _pipeline_case(V=8192, K=200, B=2, W=6, dtype_cfg="cfg1", **scaled):
+    return wk.CONFIGS[dtype_cfg].scaled(B=B, W=W, V=V, top_k=K, **scaled)
+
+
+def test_pipeline_rows_with_few_finite_logits_and_an_infinite_logit():
+    from gpu_harness import check_parity, oracle_prime, step_kwargs
+    wl = _pipeline_case()
+    inp = wk.make_step_inputs(wl)
+    inp.cond[0, 0, 150:] = -np.inf           # fewer finite logits than K: the candidates cannot hold the top-K
+    inp.uncond[0, 0, 150:] = -np.inf
+    inp.cond[0, 1, :] = -np.inf              # nothing finite
+    inp.cond[0, 2, 77] = np.inf              # an infinite logit: no finite maximum
+    inp.cond[1, 3, ::3] = -np.inf
+    prev = oracle_prime(inp)
+    rep, got, ref = check_parity(inp.cond, inp.uncond, prev.tokens, prev.probs, step_kwargs(inp), inp.win_len)
+    assert got.status[0] & oracle.STATUS_DEGENERATE_ROW
+
+
+def test_pipeline_all_equal_logits_overflow_the_candidate_lists():
+    from gpu_harness import check_parity, step_kwargs
+    wl = _pipeline_case(V=4096, K=64, B=1, W=3)
+    inp = wk.make_step_inputs(wl)
+    inp.cond[:] = 0.25
+    inp.uncond[:] = 0.25
+    q = oracle.Probs.uniform(wl.B, wl.W, wl.kcap, wl.V)
+    drafts = np.array([[3, 70, 4000]], np.int32)
+    rep, got, ref = check_parity(inp.cond, inp.uncond, drafts, q, step_kwargs(inp), inp.win_len)
+    assert np.array_equal(got.ids[0, 0], np.arange(64))
+
+
+def test_pipeline_bf16_ties_at_the_threshold():
+    # few distinct values: the threshold bin holds more members than the on-chip ranking takes
+    wl = wk.CONFIGS["cfg2"].scaled(B=2, W=3, V=16384, top_k=500, sigma=0.05, peaks=0)
+    rep, got, ref, inp, prev = _run(wl)
+    assert len(np.unique(wk.bf16_bits_to_f32(inp.cond[0, 0]))) < 2000
+
+
+def test_pipeline_k1_no_guidance_and_temperature():
+    from gpu_harness import check_parity, oracle_prime, step_kwargs
+    _run(_pipeline_case(V=4096, K=1, B=2, W=5))
+    wl = wk.CONFIGS["cfg3"].scaled(B=3, V=16384, top_k=700, temperature=0.7)
+    inp = wk.make_step_inputs(wl)
+    prev = oracle_prime(inp)
+    check_parity(inp.cond, None, prev.tokens, prev.probs, step_kwargs(inp), inp.win_len)
+
+
+def test_pipeline_structured_row_defeats_the_sample():
+    # every sample tile (every 8th tile of 256) is very negative: the sampled threshold is far too low,
+    # the lists overflow and the row is redone exactly
+    from gpu_harness import check_parity, oracle_prime, step_kwargs
+    wl = _pipeline_case(V=8192, K=100, B=1, W=2)
+    inp = wk.make_step_inputs(wl)
+    for t in range(0, 32, 8):
+        inp.cond[:, :, t * 256:(t + 1) * 256] -= 50.0
+        inp.uncond[:, :, t * 256:(t + 1) * 256] -= 50.0
+    prev = oracle_prime(inp)
+    check_parity(inp.cond, inp.uncond, prev.tokens, prev.probs, step_kwargs(inp), inp.win_len)
+    # and the opposite: the sample tiles hold the largest values, so the threshold is too high
+    inp2 = wk.make_step_inputs(wl)
+    for t in range(0, 32, 8):
+        inp2.cond[:, :, t * 256:(t + 1) * 256] += 50.0
+        inp2.uncond[:, :, t * 256:(t + 1) * 256] += 50.0
+    prev2 = oracle_prime(inp2)
+    check_parity(inp2.cond, inp2.uncond, prev2.tokens, prev2.probs, step_kwargs(inp2), inp2.win_len)
