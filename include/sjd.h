@@ -55,8 +55,10 @@ extern "C" {
 #define SJD_FLAG_DRAFT_ALL 2 /* no verification: draw every valid row from its own p (initial drafts; Section
                                 4.2 strategies that sample from a predicted distribution).  accept_len = 0. */
 
-#define SJD_FLAG_FORCE_GENERIC 4 /* diagnostics: use the any-shape multi-pass row kernel even where the
-                                   single-pass streaming kernel applies (results are identical)          */
+#define SJD_FLAG_FORCE_GENERIC 4 /* diagnostics: use the any-shape multi-pass row kernel even where a
+                                   single-pass kernel applies (results are identical)                    */
+#define SJD_FLAG_FORCE_TILES 8   /* diagnostics: skip the single-pass kernel that cuts a row into one id
+                                   range per thread; the tile-dealing one is used where it applies        */
 
 /* cnt value of a row of sjd_probs that stands for the uniform distribution over V (1/V each); used for
  * window slots that were initialised at random and have no previous-iteration distribution. */

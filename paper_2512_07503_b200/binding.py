@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 SJD_F32, SJD_BF16 = 0, 1
-SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL, SJD_FLAG_FORCE_GENERIC = 1, 2, 4
+SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL, SJD_FLAG_FORCE_GENERIC, SJD_FLAG_FORCE_TILES = 1, 2, 4, 8
 SJD_Q_UNIFORM = -1
 SJD_OUT_INVALID, SJD_OUT_ACCEPTED, SJD_OUT_RESIDUAL, SJD_OUT_REUSED, SJD_OUT_RESAMPLED = 0, 1, 2, 3, 4
 SJD_STATUS_QTOK_NONPOSITIVE, SJD_STATUS_EMPTY_RESIDUAL, SJD_STATUS_DEGENERATE_ROW = 1, 2, 4

@@ -185,30 +185,44 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   return v;
 }
 
-// Merged logits y of the lane's eight elements of a staged tile, as four packed pairs:
-// d = c - u; g = fma(s, d, u); y = g * inv_T, one rounding per operation.  Multiplying by 1.0f is exact,
-// so the last step is skipped when inv_T == 1.  ctile / utile are shared-memory addresses.
+// A thread's share of a staged tile as it lies in shared memory: 8 logits of each array.
+template <int DTYPE>
+struct RawTile {
+  uint4 c[DTYPE == 1 ? 1 : 2];
+  uint4 u[DTYPE == 1 ? 1 : 2];
+};
+
+template <int DTYPE, bool has_u>
+__device__ __forceinline__ void load_raw(uint32_t ctile, uint32_t utile, int lane, RawTile<DTYPE>& r) {
+  r.c[0] = lds128(ctile + lane * 16);
+  if (DTYPE != 1) r.c[DTYPE == 1 ? 0 : 1] = lds128(ctile + 512 + lane * 16);
+  if (has_u) {
+    r.u[0] = lds128(utile + lane * 16);
+    if (DTYPE != 1) r.u[DTYPE == 1 ? 0 : 1] = lds128(utile + 512 + lane * 16);
+  }
+}
+
+// Merged logits y of the thread's eight elements, as four packed pairs: d = c - u; g = fma(s, d, u);
+// y = g * inv_T, one rounding per operation.  Multiplying by 1.0f is exact, so the last step is skipped
+// when inv_T == 1.
 template <int DTYPE, bool has_u, bool has_t>
-__device__ __forceinline__ void tile_y8(uint32_t ctile, uint32_t utile, int lane, uint64_t s2, uint64_t t2,
-                                        float (&y)[8]) {
+__device__ __forceinline__ void merge_raw(const RawTile<DTYPE>& r, uint64_t s2, uint64_t t2, float (&y)[8]) {
   uint64_t c[4], u[4];
   if (DTYPE == 1) {
-    const uint4 w = lds128(ctile + lane * 16);
+    const uint4 w = r.c[0];
     c[0] = pack2(bf16_lo(w.x), bf16_hi(w.x)); c[1] = pack2(bf16_lo(w.y), bf16_hi(w.y));
     c[2] = pack2(bf16_lo(w.z), bf16_hi(w.z)); c[3] = pack2(bf16_lo(w.w), bf16_hi(w.w));
     if (has_u) {
-      const uint4 v = lds128(utile + lane * 16);
+      const uint4 v = r.u[0];
       u[0] = pack2(bf16_lo(v.x), bf16_hi(v.x)); u[1] = pack2(bf16_lo(v.y), bf16_hi(v.y));
       u[2] = pack2(bf16_lo(v.z), bf16_hi(v.z)); u[3] = pack2(bf16_lo(v.w), bf16_hi(v.w));
     }
   } else {
-    const uint4 a = lds128(ctile + lane * 16);
-    const uint4 b = lds128(ctile + 512 + lane * 16);
+    const uint4 a = r.c[0], b = r.c[DTYPE == 1 ? 0 : 1];
     c[0] = (uint64_t)a.x | ((uint64_t)a.y << 32); c[1] = (uint64_t)a.z | ((uint64_t)a.w << 32);
     c[2] = (uint64_t)b.x | ((uint64_t)b.y << 32); c[3] = (uint64_t)b.z | ((uint64_t)b.w << 32);
     if (has_u) {
-      const uint4 p = lds128(utile + lane * 16);
-      const uint4 q = lds128(utile + 512 + lane * 16);
+      const uint4 p = r.u[0], q = r.u[DTYPE == 1 ? 0 : 1];
       u[0] = (uint64_t)p.x | ((uint64_t)p.y << 32); u[1] = (uint64_t)p.z | ((uint64_t)p.w << 32);
       u[2] = (uint64_t)q.x | ((uint64_t)q.y << 32); u[3] = (uint64_t)q.z | ((uint64_t)q.w << 32);
     }
@@ -220,6 +234,14 @@ __device__ __forceinline__ void tile_y8(uint32_t ctile, uint32_t utile, int lane
     if (has_t) g = mul2(g, t2);
     unpack2(g, y[2 * k], y[2 * k + 1]);
   }
+}
+
+template <int DTYPE, bool has_u, bool has_t>
+__device__ __forceinline__ void tile_y8(uint32_t ctile, uint32_t utile, int lane, uint64_t s2, uint64_t t2,
+                                        float (&y)[8]) {
+  RawTile<DTYPE> r;
+  load_raw<DTYPE, has_u>(ctile, utile, lane, r);
+  merge_raw<DTYPE, has_u, has_t>(r, s2, t2, y);
 }
 
 // ---------------------------------------------------------------------------------------------------

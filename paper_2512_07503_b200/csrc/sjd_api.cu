@@ -12,6 +12,7 @@
 #include "device_utils.cuh"
 #include "row_kernels.cuh"
 #include "rows_pipeline.cuh"
+#include "rows_ranges.cuh"
 #include "verify_kernel.cuh"
 #include "advance_kernel.cuh"
 
@@ -96,6 +97,85 @@ bool plan_pipeline(const sjd_params* P, int kcap, sjd::PipeCfg* cfg, size_t* sme
     return true;
   }
   return false;
+}
+
+// ---- the kernel with one id range per filter thread (rows_ranges.cuh) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled through the runtime (no link against the driver library); nullptr when unavailable.
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess ||
+        qr != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// Same sampling rule as plan_pipeline; the sample is stage 0, i.e. 1/S of the row.
+bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem) {
+  const int V = P->V;
+  const int es = P->logits_dtype == SJD_BF16 ? 2 : 4;
+  const int bw = 64 / es;  // elements per stage and range
+  if (kcap > sjd::kKcapMax || V % sjd::kRangeThreads != 0) return false;
+  const int R = V / sjd::kRangeThreads;
+  if (R % bw != 0) return false;
+  const int S = R / bw;
+  if (S < 2 || S > 16) return false;
+  // all rows must lie at one pitch: row r = b W + i starts at r * stride_w
+  if (P->B > 1 && P->stride_b != (int64_t)P->W * P->stride_w) return false;
+  if ((int64_t)P->B * P->W >= (1ll << 31)) return false;
+  const int mask_words = (R / 2 + 31) / 32;
+  if (mask_words > sjd::kMaskWordsMax) return false;
+  const int n_sample = sjd::kRangeThreads * bw;
+  const double a = (double)kcap / S;
+  const double root = 1.75 + std::sqrt(1.75 * 1.75 + a);
+  const int m = (int)std::ceil(root * root);
+  if (m > n_sample / 2 || m > n_sample / 8) return false;  // the rank must exist among the group maxima too
+  const double mean = (double)m * S, sd = (double)S * std::sqrt((double)m);
+  if (mean + 4.0 * sd > (double)sjd::kRangeDenseCap) return false;
+  const double per_thread = (mean * (S - 1) / S + 2.1 * m) / sjd::kRangeThreads;  // pair entries, sample kept against a floor
+  if (per_thread + 5.0 * std::sqrt(per_thread) + 1.0 > (double)(sjd::kListCap - 4)) return false;
+  if (encode_tiled_fn() == nullptr) return false;
+  cfg->sample_rank = m;
+  cfg->stages = S;
+  cfg->range_len = R;
+  cfg->mask_words = mask_words;
+  *smem = sjd::range_smem_bytes(mask_words);
+  return *smem <= kSmemLimit;
+}
+
+// Tensor map over one logits array: dims {R ids, 256 ranges, rows}, box {64 bytes, 256, 1}, 64-byte swizzle.
+bool make_range_map(CUtensorMap* map, const void* base, const sjd_params* P, const sjd::RangeCfg& cfg) {
+  const int es = P->logits_dtype == SJD_BF16 ? 2 : 4;
+  const cuuint64_t dims[3] = {(cuuint64_t)cfg.range_len, (cuuint64_t)sjd::kRangeThreads, (cuuint64_t)P->B * (cuuint64_t)P->W};
+  const cuuint64_t strides[2] = {(cuuint64_t)cfg.range_len * es, (cuuint64_t)P->stride_w * es};
+  const cuuint32_t box[3] = {(cuuint32_t)(64 / es), (cuuint32_t)sjd::kRangeThreads, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = encode_tiled_fn()(map, P->logits_dtype == SJD_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                       3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                       CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int DTYPE>
+cudaError_t launch_ranges(const sjd::RowArgs& ra, const sjd::RangeCfg& cfg, const CUtensorMap& mc, const CUtensorMap& mu,
+                          size_t smem, int grid, cudaStream_t st) {
+  auto kern = sjd::rows_ranges_kernel<DTYPE, kFinisherWarps>;
+  static bool configured = false;  // per instantiation; the attribute is sticky for the process
+  if (!configured) {
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  kern<<<grid, (8 + kFinisherWarps + 1) * 32, smem, st>>>(ra, cfg, mc, mu);
+  return cudaGetLastError();
 }
 
 template <int DTYPE>
@@ -230,9 +310,17 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
   }
   {
     sjd::PipeCfg cfg;
+    sjd::RangeCfg rcfg;
     size_t smem = 0;
     cudaError_t e;
-    if (!(P->flags & SJD_FLAG_FORCE_GENERIC) && plan_pipeline(P, kcap, &cfg, &smem)) {
+    CUtensorMap map_c, map_u;
+    const bool fast = !(P->flags & (SJD_FLAG_FORCE_GENERIC | SJD_FLAG_FORCE_TILES));
+    if (fast && plan_ranges(P, kcap, &rcfg, &smem) && make_range_map(&map_c, logits_cond, P, rcfg) &&
+        make_range_map(&map_u, logits_uncond ? logits_uncond : logits_cond, P, rcfg)) {
+      const int grid = rows < sm_count() ? rows : sm_count();
+      e = P->logits_dtype == SJD_BF16 ? launch_ranges<1>(ra, rcfg, map_c, map_u, smem, grid, stream)
+                                      : launch_ranges<0>(ra, rcfg, map_c, map_u, smem, grid, stream);
+    } else if (!(P->flags & SJD_FLAG_FORCE_GENERIC) && plan_pipeline(P, kcap, &cfg, &smem)) {
       const int grid = rows < sm_count() ? rows : sm_count();
       e = P->logits_dtype == SJD_BF16 ? launch_pipeline<1>(ra, cfg, smem, grid, stream)
                                       : launch_pipeline<0>(ra, cfg, smem, grid, stream);
