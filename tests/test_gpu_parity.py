@@ -207,3 +207,10 @@ def test_pipeline_structured_row_defeats_the_sample():
         inp2.uncond[:, :, t * 256:(t + 1) * 256] += 50.0
     prev2 = oracle_prime(inp2)
     check_parity(inp2.cond, inp2.uncond, prev2.tokens, prev2.probs, step_kwargs(inp2), inp2.win_len)
+
+
+@pytest.mark.parametrize("force", [4, 8])  # SJD_FLAG_FORCE_GENERIC, SJD_FLAG_FORCE_TILES
+def test_every_row_kernel_gives_the_same_answer(force):
+    # the same shapes through the any-shape kernel and the tile-dealing kernel instead of the range kernel
+    _run(wk.CONFIGS["cfg2"].scaled(W=6), flags=oracle.FLAG_REUSE | force)
+    _run(wk.CONFIGS["cfg3"].scaled(B=6), flags=oracle.FLAG_REUSE | force)
