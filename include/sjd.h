@@ -124,7 +124,7 @@ typedef struct {
   void* ev_rows_end;          /* ... and just after it (tracing; NULL = not recorded)                      */
 } sjd_params;
 
-/* Library version (SJD_VERSION of the build). */
+/* Library version (the SJD_VERSION the library was compiled with). */
 int sjd_version(void);
 
 /* Static text for a return code. */

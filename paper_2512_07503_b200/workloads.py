@@ -4,7 +4,7 @@ This module holds NONE of the method's arithmetic: it only draws Gaussian logits
 the storage type and lays out the window bookkeeping.  Both the CUDA path and the CPU oracle consume
 what it returns, so that the two see the same bits.
 
-The five workloads follow the benchmark definition of the build (top-K 2000 and guidance weight 3.0
+The workloads are the benchmark's configurations (top-K 2000 and guidance weight 3.0
 are the paper's Section 5.1 settings; window sizes 16-64 lie in the range of the paper's window
 ablation; 576 tokens is the 24x24 grid the paper quotes for Janus-Pro).  They stand in for the
 paper's prompt sets and models, none of which can be used offline.
