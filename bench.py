@@ -40,6 +40,10 @@ def parse_args():
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--init-mode", type=int, default=0, choices=[0, 1, 2, 3, 4],
+                    help="--loop only: token initialisation (0 random, 1 repeat left, 2 repeat above, 3 sample left, 4 sample above)")
+    ap.add_argument("--loop-source", default="markov", choices=["markov", "stripes"],
+                    help="--loop only: synthetic logit source (first-order Markov chain, or an image of vertical stripes)")
     ap.add_argument("--loop", action="store_true",
                     help="run the full decode loop of the 48x48 grid workload (cfg5) instead of the single-step benchmark")
     return ap.parse_args()
@@ -441,9 +445,21 @@ def run_loop(args):
     noise_c = torch.randn(N, V, generator=g, device=dev).to(torch.bfloat16)
     g.manual_seed(6)
     noise_u = torch.randn(N, V, generator=g, device=dev).to(torch.bfloat16)
+    G = 48
     dl = DecodeLoop(batch=1, window=W, vocab=V, n_total=N, logits_dtype=torch.bfloat16, top_k=K, cfg_scale=3.0, seed=5,
-                    device=dev)
+                    init_mode=args.init_mode, grid_width=G, device=dev)
     ar = torch.arange(W, device=dev)
+    g.manual_seed(8)
+    colours = torch.randperm(V, generator=g, device=dev)[:G]
+
+    def stripes(d):
+        # every column of the grid has its own colour: the prediction is peaked on it whatever the prefix is
+        pos = (d.pos_base[0] + ar).clamp(max=N - 1)
+        cond = 0.3 * noise_c[pos].float()
+        cond[ar, colours[pos % G]] += 16.0
+        cond_s = cond.to(torch.bfloat16)
+        unc_s = (cond_s.float() + 0.3 * noise_u[pos].float()).to(torch.bfloat16)
+        return cond_s.view(1, W, V), unc_s.view(1, W, V)
 
     def source(d):
         p0 = int(d.pos_base[0].item())
@@ -462,7 +478,7 @@ def run_loop(args):
     t0 = time.perf_counter()
     lib_ms = 0.0
     while not dl.done():
-        cond, unc = source(dl)
+        cond, unc = stripes(dl) if args.loop_source == "stripes" else source(dl)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         dl.step(cond, unc)
@@ -471,8 +487,9 @@ def run_loop(args):
     torch.cuda.synchronize()
     wall = time.perf_counter() - t0
     lib_ms = sum(a.elapsed_time(b) for a, b in ev)
-    print(json.dumps({"workload": "cfg5: decode loop, 2304 tokens, V=65536, W=32, bf16, CFG 3.0, top-K 2000, Markov source",
-                      "steps": dl.steps, "tokens": N, "mean_committed_per_step": round(N / dl.steps, 4),
+    print(json.dumps({"workload": "cfg5: decode loop, 2304 tokens, V=65536, W=32, bf16, CFG 3.0, top-K 2000, "
+                                  + ("Markov source" if args.loop_source == "markov" else "vertical-stripes source"),
+                      "init_mode": args.init_mode, "grid_width": G, "steps": dl.steps, "tokens": N, "mean_committed_per_step": round(N / dl.steps, 4),
                       "step_compression_S": round(N / dl.steps, 4), "library_ms_total": round(lib_ms, 3),
                       "library_us_per_step": round(1e3 * lib_ms / dl.steps, 2), "wall_s_including_logit_source": round(wall, 3),
                       "complete": bool((dl.committed >= 0).all().item())}), flush=True)

@@ -97,6 +97,13 @@ typedef struct {
   int32_t* cnt;    /* [B,W]       entries used (kcap for a valid row), or SJD_Q_UNIFORM on input             */
 } sjd_probs;
 
+/* Token initialisation of new window slots (Section 4.2, "Token Initialization with Spatial Prior"). */
+#define SJD_INIT_RANDOM 0        /* uniform token, uniform reference distribution (vanilla Jacobi decoding) */
+#define SJD_INIT_REPEAT_LEFT 1   /* strategy (a): the token of the left neighbour, position p-1            */
+#define SJD_INIT_REPEAT_ABOVE 2  /* strategy (b): the token of the neighbour above, position p-G           */
+#define SJD_INIT_SAMPLE_LEFT 3   /* strategy (c): a draw from the prediction made for the left neighbour   */
+#define SJD_INIT_SAMPLE_ABOVE 4  /* strategy (d): a draw from the prediction made for the neighbour above  */
+
 /* HOST struct, read during the call; device pointers inside it are read by the kernels. */
 typedef struct {
   int32_t struct_size;        /* sizeof(sjd_params)                                                        */
@@ -122,6 +129,8 @@ typedef struct {
   void* stream;               /* cudaStream_t the work is enqueued on (NULL = legacy default stream)       */
   void* ev_rows_begin;        /* optional cudaEvent_t recorded on `stream` just before the row stage ...   */
   void* ev_rows_end;          /* ... and just after it (tracing; NULL = not recorded)                      */
+  int32_t init_mode;          /* SJD_INIT_*: how the window functions fill new slots; sjd_step ignores it  */
+  int32_t grid_width;         /* G: tokens per image row of the raster grid (the "above" strategies), >= 1 */
 } sjd_params;
 
 /* Library version (the SJD_VERSION the library was compiled with). */
@@ -167,9 +176,13 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
  * of Step 3 "accepted tokens are appended", the last sentence of Step 4 "accepted and reinitialised tokens
  * form the next window"; random initialisation is the baseline of Section 4.2).
  *
- * sjd_window_init() fills the first window: drafts[b,i] for i < win_len[b] is a token drawn uniformly from
- * [0,V) (Philox purpose 4, counter = (pos_base[b]+i, seq_base+b, iteration[b], 4), token = floor(x0 V / 2^32))
- * and its reference distribution is SJD_Q_UNIFORM with tok_prob = 1/V; rows beyond win_len get token -1.
+ * sjd_window_init() fills the first window.  With SJD_INIT_RANDOM drafts[b,i] for i < win_len[b] is a token
+ * drawn uniformly from [0,V) (Philox purpose 4, counter = (pos_base[b]+i, seq_base+b, iteration[b], 4), token =
+ * floor(x0 V / 2^32)) and its reference distribution is SJD_Q_UNIFORM with tok_prob = 1/V; rows beyond win_len
+ * get token -1.  With a spatial-prior mode, slot i copies slot i-1 ("left" modes, and "above" modes for
+ * i < G) or slot i-G ("above" modes); a copied token is a deterministic draft, so its reference distribution
+ * is the point mass on it (cnt 1, vals[0] = tok_prob = 1); slot 0 is random as above.  There are no
+ * predictions yet, so the two sampling modes act as their repeating counterparts here.
  *
  * sjd_window_advance() takes what sjd_step() just produced (accept_len, out_tokens, out_probs) and
  *   - commits c_b tokens per sequence: the accepted prefix plus the residual draw at the first rejected row
@@ -178,10 +191,24 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
  *     n_committed[b] when that is not NULL;
  *   - builds the next window in next_drafts / next_probs (which must not alias the step's outputs): row i takes
  *     the step's row i+c with that row's distribution as its reference when i+c < win_len, else a newly
- *     initialised token as in sjd_window_init() with the iteration index of the step that just ran;
+ *     initialised token, with the iteration index of the step that just ran in the generator's counter:
+ *       SJD_INIT_RANDOM        as in sjd_window_init();
+ *       SJD_INIT_REPEAT_LEFT   the token at position p-1, point-mass reference;
+ *       SJD_INIT_REPEAT_ABOVE  the token at position p-G (p-1 when p < G), point-mass reference.  The token at an
+ *                              earlier position is the committed one before the verified window, the step's
+ *                              output token inside it, and a new slot's own initial token after it;
+ *       SJD_INIT_SAMPLE_LEFT   a draw from the distribution of the last verified row (the nearest prediction to
+ *                              the left), which also becomes the reference; fixed-point inverse CDF on Philox
+ *                              purpose 5, counter = (p, seq_base+b, iteration, 5), R = x0 | x1 << 32;
+ *       SJD_INIT_SAMPLE_ABOVE  the same from the row of position p-G, stepping a further G back while that
+ *                              position is itself a new slot; when it was verified before this step (its
+ *                              distribution is gone) the committed token there with a point-mass reference;
+ *                              when p < G (or the walk leaves the grid) as SJD_INIT_SAMPLE_LEFT.
+ *     The paper names the strategies; the reference distributions, the fall-backs and the generator words are
+ *     this library's;
  *   - updates win_len, pos_base, iteration in place: pos_base += c, win_len = min(W, n_total - pos_base),
  *     iteration += 1.  A sequence is finished when its win_len is 0.
- * params supplies B, W, V, top_k, seq_base and stream; its win_len/pos_base/iteration fields are not used
+ * params supplies B, W, V, top_k, seq_base, init_mode, grid_width and stream; its win_len/pos_base/iteration fields are not used
  * (the arrays are passed explicitly because they are written).  All pointers are device pointers.  Both
  * calls are asynchronous on params->stream and return SJD_OK or a negative SJD_ERR_*.
  */

@@ -17,6 +17,7 @@ from . import build as _build
 SJD_F32, SJD_BF16 = 0, 1
 SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL, SJD_FLAG_FORCE_GENERIC, SJD_FLAG_FORCE_TILES = 1, 2, 4, 8
 SJD_Q_UNIFORM = -1
+SJD_INIT_RANDOM, SJD_INIT_REPEAT_LEFT, SJD_INIT_REPEAT_ABOVE, SJD_INIT_SAMPLE_LEFT, SJD_INIT_SAMPLE_ABOVE = 0, 1, 2, 3, 4
 SJD_OUT_INVALID, SJD_OUT_ACCEPTED, SJD_OUT_RESIDUAL, SJD_OUT_REUSED, SJD_OUT_RESAMPLED = 0, 1, 2, 3, 4
 SJD_STATUS_QTOK_NONPOSITIVE, SJD_STATUS_EMPTY_RESIDUAL, SJD_STATUS_DEGENERATE_ROW = 1, 2, 4
 SJD_W_MAX = 512
@@ -34,7 +35,7 @@ class sjd_params(C.Structure):
                 ("win_len", C.c_void_p), ("pos_base", C.c_void_p), ("iteration", C.c_void_p),
                 ("out_flags", C.c_void_p), ("status", C.c_void_p), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p), ("ev_rows_begin", C.c_void_p),
-                ("ev_rows_end", C.c_void_p)]
+                ("ev_rows_end", C.c_void_p), ("init_mode", C.c_int32), ("grid_width", C.c_int32)]
 
 
 class SjdError(RuntimeError):
@@ -134,7 +135,8 @@ def make_params(logits: torch.Tensor, *, top_k: int, cfg_scale: float = 1.0, inv
                 win_len: Optional[torch.Tensor] = None, pos_base: Optional[torch.Tensor] = None,
                 iteration: Optional[torch.Tensor] = None, out_flags: Optional[torch.Tensor] = None,
                 status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-                stream: Optional[torch.cuda.Stream] = None, seq_base: int = 0) -> sjd_params:
+                stream: Optional[torch.cuda.Stream] = None, seq_base: int = 0, init_mode: int = 0,
+                grid_width: int = 1) -> sjd_params:
     """Fill an ``sjd_params`` from a [B,W,V] logits tensor (fp32 or bf16, vocabulary axis contiguous)."""
     if logits.dim() != 3 or logits.stride(2) != 1:
         raise SjdError("logits must be [B,W,V] with a contiguous vocabulary axis")
@@ -157,6 +159,8 @@ def make_params(logits: torch.Tensor, *, top_k: int, cfg_scale: float = 1.0, inv
     p.flags = flags
     p.iteration0 = iteration0
     p.seq_base = seq_base
+    p.init_mode = init_mode
+    p.grid_width = grid_width
     p.win_len = _opt_ptr(win_len)
     p.pos_base = _opt_ptr(pos_base)
     p.iteration = _opt_ptr(iteration)

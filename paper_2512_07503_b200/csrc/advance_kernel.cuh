@@ -1,8 +1,10 @@
 // Window bookkeeping between two Jacobi iterations (paper Section 4.1, Step 1 and the closing sentence of
 // Step 4): the accepted prefix and the residual token are committed, the rows that remain unaccepted move
 // to the front of the window and keep this iteration's distributions as their verification reference,
-// and the freed slots are filled with newly initialised tokens (random initialisation, Section 4.2's
-// baseline) whose reference distribution is uniform.
+// and the freed slots are filled with newly initialised tokens: random ones whose reference distribution
+// is uniform (Section 4.2's baseline), or one of the four spatial-prior strategies of Section 4.2 - the
+// token of the left or above neighbour on the raster grid (a deterministic draft: point-mass reference),
+// or a draw from the prediction the step just made for that neighbour (that prediction is the reference).
 #pragma once
 
 #include "device_utils.cuh"
@@ -10,10 +12,14 @@
 namespace sjd {
 
 constexpr int kPurposeTokenInit = 4;  // Philox purpose of a randomly initialised draft token
+constexpr int kPurposePriorInit = 5;  // Philox purpose of a draft drawn from a neighbour's prediction
+
+constexpr int kInitRandom = 0, kInitRepeatLeft = 1, kInitRepeatAbove = 2, kInitSampleLeft = 3, kInitSampleAbove = 4;
 
 struct AdvanceArgs {
   int B, W, V, kcap, n_total;
   int seq_base;
+  int init_mode, grid_width;
   uint32_t seed_lo, seed_hi;
   // result of the step that just ran
   const int32_t* accept_len;
@@ -87,11 +93,65 @@ __global__ void __launch_bounds__(NT) advance_rows_kernel(const AdvanceArgs a) {
       a.next_tok_prob[row] = a.step_tok_prob[srow];
       a.next_cnt[row] = n;
     }
-  } else if (threadIdx.x == 0) {
-    // a new slot: random token, uniform reference distribution
-    a.next_drafts[row] = random_token(pos1 + i, a.seq_base + b, iter, a.V, a.seed_lo, a.seed_hi);
-    a.next_tok_prob[row] = __fdiv_rn(1.0f, (float)a.V);
-    a.next_cnt[row] = -1;
+    return;
+  }
+  // a new slot at absolute position p
+  const int p = pos1 + i;
+  const int G = a.grid_width;
+  const int end0 = pos0 + L;  // first position after the verified window
+  const int mode = a.init_mode;
+  const bool above = (mode == kInitRepeatAbove || mode == kInitSampleAbove) && p >= G;
+  const bool sample = mode == kInitSampleLeft || mode == kInitSampleAbove;
+  if (mode == kInitRandom || L < 1) {
+    if (threadIdx.x == 0) {
+      a.next_drafts[row] = random_token(p, a.seq_base + b, iter, a.V, a.seed_lo, a.seed_hi);
+      a.next_tok_prob[row] = __fdiv_rn(1.0f, (float)a.V);
+      a.next_cnt[row] = -1;
+    }
+    return;
+  }
+  // the position whose token (repeat) or prediction (sample) initialises this slot
+  int r;
+  if (!sample) {
+    // positions at or after end0 are new slots themselves: follow their own rule back into known tokens
+    r = above ? p - G : p - 1;
+    while (r >= end0) r -= (mode == kInitRepeatAbove && r >= G) ? G : 1;
+  } else if (above) {
+    r = p - G;
+    while (r >= end0) r -= G;
+    if (r < 0) r = end0 - 1;  // left the grid: the last verified row, as for "sample left"
+  } else {
+    r = end0 - 1;
+  }
+  if (!sample || r < pos0) {
+    if (threadIdx.x == 0) {
+      const int tok = r < pos0 ? a.committed[(size_t)b * a.n_total + r] : a.step_tokens[(size_t)b * a.W + (r - pos0)];
+      a.next_drafts[row] = tok;
+      a.next_tok_prob[row] = 1.0f;
+      nid[0] = tok;
+      nv[0] = 1.0f;
+      a.next_cnt[row] = 1;
+    }
+    return;
+  }
+  // draw from the prediction of row r - pos0 and keep that prediction as the reference
+  __shared__ uint64_t scratch[2 * (NT / 32) + 4];
+  const size_t srow = (size_t)b * a.W + (r - pos0);
+  const int32_t* sid = a.step_ids + srow * a.kcap;
+  const float* sv = a.step_vals + srow * a.kcap;
+  const int n = min(max(a.step_cnt[srow], 0), a.kcap);
+  for (int k = threadIdx.x; k < n; k += NT) {
+    nid[k] = sid[k];
+    nv[k] = sv[k];
+  }
+  const Philox4 rnd = philox4x32_10((uint32_t)p, (uint32_t)(a.seq_base + b), (uint32_t)iter, kPurposePriorInit,
+                                    a.seed_lo, a.seed_hi);
+  int k = group_icdf<NT, 0>([&](int j) { return fixed_weight(sv[j]); }, n, random64(rnd), threadIdx.x, scratch);
+  if (k < 0) k = 0;
+  if (threadIdx.x == 0) {
+    a.next_drafts[row] = n > 0 ? sid[k] : 0;
+    a.next_tok_prob[row] = n > 0 ? sv[k] : 0.0f;
+    a.next_cnt[row] = n;
   }
 }
 
@@ -109,20 +169,32 @@ __global__ void advance_state_kernel(const AdvanceArgs a) {
   if (a.n_committed) a.n_committed[b] = c;
 }
 
-// First window of a sequence: every slot randomly initialised.
+// First window of a sequence.  With a spatial-prior strategy slot i copies slot i-1 (the "left" strategies,
+// and the "above" ones in the first grid row) or slot i-G; either way the chain ends at slot 0, whose
+// token is random, so every slot holds that token.  No prediction exists yet, so the sampling strategies
+// repeat as well.  With the random strategy every slot gets its own uniform token.
 __global__ void init_window_kernel(const AdvanceArgs a) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= a.B * a.W) return;
   const int b = r / a.W, i = r - b * a.W;
   const int L = min(max(a.win_len[b], 0), a.W);
-  if (i < L) {
-    a.next_drafts[r] = random_token(a.pos_base[b] + i, a.seq_base + b, a.iteration[b], a.V, a.seed_lo, a.seed_hi);
-    a.next_tok_prob[r] = __fdiv_rn(1.0f, (float)a.V);
-    a.next_cnt[r] = -1;
-  } else {
+  if (i >= L) {
     a.next_drafts[r] = -1;
     a.next_tok_prob[r] = 0.0f;
     a.next_cnt[r] = 0;
+    return;
+  }
+  const int src = a.init_mode == kInitRandom ? i : 0;
+  const int tok = random_token(a.pos_base[b] + src, a.seq_base + b, a.iteration[b], a.V, a.seed_lo, a.seed_hi);
+  a.next_drafts[r] = tok;
+  if (a.init_mode == kInitRandom || i == 0) {
+    a.next_tok_prob[r] = __fdiv_rn(1.0f, (float)a.V);
+    a.next_cnt[r] = -1;
+  } else {
+    a.next_tok_prob[r] = 1.0f;
+    a.next_ids[(size_t)r * a.kcap] = tok;
+    a.next_vals[(size_t)r * a.kcap] = 1.0f;
+    a.next_cnt[r] = 1;
   }
 }
 

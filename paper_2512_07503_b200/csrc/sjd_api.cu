@@ -398,11 +398,15 @@ int fill_advance(sjd::AdvanceArgs* a, const sjd_params* P, int32_t n_total, uint
   if (P->struct_size != (int32_t)sizeof(sjd_params)) return SJD_ERR_STRUCT;
   if (!win_len || !pos_base || !iteration || !next_drafts || check_probs(next_probs) != SJD_OK) return SJD_ERR_NULL;
   if (P->B < 0 || P->W < 1 || P->W > SJD_W_MAX || P->V < 1 || P->top_k < 1 || n_total < 0) return SJD_ERR_SHAPE;
+  if (P->init_mode < SJD_INIT_RANDOM || P->init_mode > SJD_INIT_SAMPLE_ABOVE) return SJD_ERR_SHAPE;
+  if (P->init_mode != SJD_INIT_RANDOM && P->grid_width < 1) return SJD_ERR_SHAPE;
   std::memset(a, 0, sizeof(*a));
   a->B = P->B; a->W = P->W; a->V = P->V;
   a->kcap = P->top_k < P->V ? P->top_k : P->V;
   a->n_total = n_total;
   a->seq_base = P->seq_base;
+  a->init_mode = P->init_mode;
+  a->grid_width = P->grid_width > 0 ? P->grid_width : 1;
   a->seed_lo = (uint32_t)(seed & 0xffffffffu);
   a->seed_hi = (uint32_t)(seed >> 32);
   a->win_len = win_len; a->pos_base = pos_base; a->iteration = iteration;

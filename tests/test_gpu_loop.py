@@ -13,17 +13,19 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64):
+def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64, init_mode=0, grid_width=1, windows=False):
     from paper_2512_07503_b200.decode import DecodeLoop
     src = wk.MarkovSource(V, N, dtype, states=states)
     flags = oracle.FLAG_REUSE if reuse else 0
+    trace = []
     ref_committed, ref_steps, ref_counts = loop.decode(
         lambda w: src.logits(w.drafts, w.win_len, w.pos_base, w.committed), B=B, W=W, V=V, n_total=N, dtype=dtype,
-        top_k=top_k, cfg_scale=3.0, flags=flags, seed=seed, n_threads=8)
+        top_k=top_k, cfg_scale=3.0, flags=flags, seed=seed, n_threads=8, init_mode=init_mode, grid_width=grid_width,
+        trace=trace)
 
     tdt = torch.bfloat16 if dtype == wk.BF16 else torch.float32
     dl = DecodeLoop(batch=B, window=W, vocab=V, n_total=N, logits_dtype=tdt, top_k=top_k, cfg_scale=3.0, reuse=reuse,
-                    seed=seed, device=DEV)
+                    seed=seed, init_mode=init_mode, grid_width=grid_width, device=DEV)
 
     def up(a):
         if dtype == wk.BF16:
@@ -31,6 +33,8 @@ def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64):
         return torch.from_numpy(a).to(DEV)
 
     def source(d):
+        if windows:
+            _same_window(d, trace[d.steps][0])
         c, u = src.logits(d.window_tokens.cpu().numpy(), d.win_len.cpu().numpy(), d.pos_base.cpu().numpy(),
                           d.committed.cpu().numpy())
         return up(c), up(u)
@@ -38,6 +42,40 @@ def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64):
     committed, steps, counts = dl.run(source, max_steps=4 * N)
     assert int(dl.status.max().item()) & 8 == 0
     return (committed.numpy(), steps, counts.numpy()), (ref_committed, ref_steps, ref_counts)
+
+
+def _same_window(d, w):
+    """The device loop's current window against the oracle's: drafts, reference distributions, state."""
+    L = w.win_len
+    assert np.array_equal(d.win_len.cpu().numpy(), L) and np.array_equal(d.pos_base.cpu().numpy(), w.pos_base)
+    q = d.q[d.cur]
+    drafts, cnt, tp = d.window_tokens.cpu().numpy(), q.cnt.cpu().numpy(), q.tok_prob.cpu().numpy()
+    ids, vals = q.ids.cpu().numpy(), q.vals.cpu().numpy()
+    for b in range(L.shape[0]):
+        n = int(L[b])
+        assert np.array_equal(drafts[b, :n], w.drafts[b, :n]), (b, drafts[b, :n], w.drafts[b, :n])
+        assert np.array_equal(cnt[b, :n], w.probs.cnt[b, :n])
+        np.testing.assert_allclose(tp[b, :n], w.probs.tok_prob[b, :n], rtol=1e-5, atol=0)
+        for i in range(n):
+            k = max(int(cnt[b, i]), 0)
+            assert np.array_equal(ids[b, i, :k], w.probs.ids[b, i, :k])
+            np.testing.assert_allclose(vals[b, i, :k], w.probs.vals[b, i, :k], rtol=1e-5, atol=1e-30)
+
+
+@pytest.mark.parametrize("mode", [1, 2, 3, 4])
+@pytest.mark.parametrize("B,W,V,N,K,dtype,G", [(2, 8, 4096, 60, 64, wk.F32, 5), (2, 12, 8192, 70, 300, wk.BF16, 16),
+                                               (1, 6, 512, 30, 40, wk.F32, 2)])
+def test_spatial_prior_initialisation_matches_the_oracle(B, W, V, N, K, dtype, G, mode):
+    # Section 4.2's four strategies, window by window: new slots' tokens and their reference distributions
+    got, ref = _both(B, W, V, N, K, dtype, init_mode=mode, grid_width=G, windows=True)
+    assert got[1] == ref[1], (got[1], ref[1])
+    assert np.array_equal(got[2], ref[2])
+    assert np.array_equal(got[0], ref[0])
+
+
+def test_random_initialisation_windows_match_the_oracle():
+    got, ref = _both(2, 8, 4096, 50, 64, wk.F32, windows=True)
+    assert np.array_equal(got[0], ref[0]) and got[1] == ref[1]
 
 
 @pytest.mark.parametrize("B,W,V,N,K,dtype,reuse", [(3, 8, 4096, 50, 64, wk.F32, True), (2, 16, 8192, 70, 300, wk.BF16, True),
