@@ -207,7 +207,7 @@ def run_ours(args):
     device = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
-    wl = wk.CONFIGS[args.workload]
+    wl = wk.workload(args.workload)
     K, Wm = args.steps, max(args.warmup, 3)
 
     # every rank owns wl.B sequences of a global batch of world * wl.B (weak scaling over sequences)
@@ -284,12 +284,17 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = run_cpu_baseline(wl, sets[0])
 
+    # status words of the last step of every input set: sequences with a row the single-pass kernel handed to
+    # the any-shape path (exact, but many times slower), and the selected row kernel
+    redone = sum(int(((d.status & 16) != 0).sum().item()) for d in sets)
+    row_kernel = ["generic", "tiles", "ranges"][sjd.sjd_row_kernel(sets[0].params)]
     if rank == 0:
         line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
                 "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(wl, world),
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-                "cpu_baseline": cpu, "hbm_gbs_whole_step": round(abytes / (ms_per_step * 1e-3) / 1e9, 1)}
+                "cpu_baseline": cpu, "hbm_gbs_whole_step": round(abytes / (ms_per_step * 1e-3) / 1e9, 1),
+                "row_kernel": row_kernel, "sequences_with_a_redone_row": redone}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -391,7 +396,7 @@ def run_reference(args):
     import oracle
     from paper_2512_07503_b200 import workloads as wk
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    wl_full = wk.CONFIGS[args.workload]
+    wl_full = wk.workload(args.workload)
     Bs = min(wl_full.B, 2)
     wl = wl_full.scaled(B=Bs)
     cores = os.cpu_count() or 1

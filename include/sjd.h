@@ -76,6 +76,8 @@ extern "C" {
 #define SJD_STATUS_EMPTY_RESIDUAL 2   /* fixed-point residual total was 0: drawn from p instead          */
 #define SJD_STATUS_DEGENERATE_ROW 4   /* a row had no finite logit: its probabilities are all 0          */
 #define SJD_STATUS_INTERNAL_TIMEOUT 8 /* a bounded on-chip wait gave up: the sequence's outputs are invalid */
+#define SJD_STATUS_ROW_REDONE 16      /* informational: a row did not fit the single-pass kernel's on-chip lists
+                                         and was redone by the any-shape path; its result is exact, the step slower */
 
 /* return codes */
 #define SJD_OK 0
@@ -147,6 +149,18 @@ uint64_t sjd_launch_count(void);
 
 /* Scratch bytes sjd_step() needs for this shape (depends on B, W only).  0 on a NULL argument. */
 size_t sjd_workspace_bytes(const sjd_params* params);
+
+/*
+ * Which row kernel sjd_step() selects for this shape and these flags (Section 3.1's sampling head has three
+ * implementations that give identical results): SJD_ROWS_RANGES, SJD_ROWS_TILES or SJD_ROWS_GENERIC, or a
+ * negative SJD_ERR_* for a shape, dtype or strides sjd_step() would refuse (pointers and the workspace are not
+ * looked at).  Decided from the shape alone: it assumes the driver offers the tensor-map encoder the range
+ * kernel needs, which every driver that runs this library's kernels does.  Launches nothing.
+ */
+#define SJD_ROWS_GENERIC 0 /* any shape: radix select over global memory, several passes                   */
+#define SJD_ROWS_TILES 1   /* V a multiple of 2,048: one pass, tiles dealt to the filter warps             */
+#define SJD_ROWS_RANGES 2  /* V a multiple of 256, kcap <= 2,048: one pass, one id range per filter thread */
+int sjd_row_kernel(const sjd_params* params);
 
 /*
  * One verify-and-redraft step (Section 4.1 Steps 3-4 on top of the Section 3.1 sampling head).

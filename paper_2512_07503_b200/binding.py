@@ -20,6 +20,7 @@ SJD_Q_UNIFORM = -1
 SJD_INIT_RANDOM, SJD_INIT_REPEAT_LEFT, SJD_INIT_REPEAT_ABOVE, SJD_INIT_SAMPLE_LEFT, SJD_INIT_SAMPLE_ABOVE = 0, 1, 2, 3, 4
 SJD_OUT_INVALID, SJD_OUT_ACCEPTED, SJD_OUT_RESIDUAL, SJD_OUT_REUSED, SJD_OUT_RESAMPLED = 0, 1, 2, 3, 4
 SJD_STATUS_QTOK_NONPOSITIVE, SJD_STATUS_EMPTY_RESIDUAL, SJD_STATUS_DEGENERATE_ROW = 1, 2, 4
+SJD_STATUS_INTERNAL_TIMEOUT, SJD_STATUS_ROW_REDONE = 8, 16
 SJD_W_MAX = 512
 
 
@@ -58,6 +59,8 @@ def lib() -> C.CDLL:
         L.sjd_launch_count.restype = C.c_uint64
         L.sjd_workspace_bytes.argtypes = [C.POINTER(sjd_params)]
         L.sjd_workspace_bytes.restype = C.c_size_t
+        L.sjd_row_kernel.argtypes = [C.POINTER(sjd_params)]
+        L.sjd_row_kernel.restype = C.c_int
         L.sjd_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs), C.POINTER(sjd_params),
                                C.c_uint64, C.c_void_p, C.c_void_p, C.POINTER(sjd_probs)]
         L.sjd_step.restype = C.c_int
@@ -128,6 +131,17 @@ def _opt_ptr(t: Optional[torch.Tensor], dtype=torch.int32) -> Optional[int]:
     if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
         raise SjdError("optional arrays must be contiguous CUDA tensors of the documented dtype")
     return t.data_ptr()
+
+
+SJD_ROWS_GENERIC, SJD_ROWS_TILES, SJD_ROWS_RANGES = 0, 1, 2
+
+
+def sjd_row_kernel(params: "sjd_params") -> int:
+    """Which row kernel sjd_step() takes for these parameters (SJD_ROWS_*)."""
+    code = lib().sjd_row_kernel(C.byref(params))
+    if code < 0:
+        _check(code)
+    return code
 
 
 def make_params(logits: torch.Tensor, *, top_k: int, cfg_scale: float = 1.0, inv_temperature: float = 1.0,

@@ -15,6 +15,7 @@ constexpr int kPurposeInit = 3;
 
 constexpr int kRowStatusDegenerate = 1;
 constexpr int kRowStatusTimeout = 2;  // a bounded on-chip wait gave up; the row has no result
+constexpr int kRowStatusRedone = 4;   // the single-pass kernel handed the row to the any-shape path (result exact)
 
 // ------------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): counter = (position, sequence, iteration, purpose),

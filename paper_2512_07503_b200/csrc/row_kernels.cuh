@@ -52,7 +52,7 @@ __device__ __forceinline__ const void* row_ptr(const void* base, int dtype, int6
 
 // One row through global memory.  All NT threads of the group call it with the same arguments.
 template <int DTYPE, int NT, int BAR>
-__device__ void row_generic(const RowArgs& a, int row, int tid, GenericSmem& sm) {
+__device__ void row_generic(const RowArgs& a, int row, int tid, GenericSmem& sm, int extra_status = 0) {
   const int b = row / a.W, i = row - b * a.W;
   const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
   RowScratch* rs = a.scratch + row;
@@ -189,7 +189,7 @@ __device__ void row_generic(const RowArgs& a, int row, int tid, GenericSmem& sm)
   if (k < 0) k = 0;
   if (tid == 0) {
     a.out_cnt[row] = kcap;
-    *rs = RowScratch{sm.p_tok, ids[k], vals[k], degenerate ? kRowStatusDegenerate : 0};
+    *rs = RowScratch{sm.p_tok, ids[k], vals[k], (degenerate ? kRowStatusDegenerate : 0) | extra_status};
   }
   group_sync<NT, BAR>();
 }

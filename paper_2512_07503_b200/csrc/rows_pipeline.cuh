@@ -871,7 +871,7 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
     if (fallback) {
       // exact any-shape path from global memory (the row is still in L2); its scratch sits on st_vals,
       // so that sel (= st_ids) stays zero
-      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals));
+      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals), kRowStatusRedone);
       continue;
     }
     // ---- normalise, write the row, draw from it ----

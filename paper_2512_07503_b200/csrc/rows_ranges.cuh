@@ -31,6 +31,7 @@ constexpr int kRangeDenseCap = 3584;        // candidates the finisher can hold 
 
 struct RangeCfg {
   int sample_rank;  // m: rank (from the top) within the sample (stage 0) that fixes tau0
+  int sample_all;   // 1: the first pass bins every sample element (m exceeds the number of groups of eight)
   int stages;       // S = R / (elements per stage and range)
   int range_len;    // R
   int mask_words;   // 32 hit bits each: R/2 pairs per range
@@ -183,7 +184,12 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
         float y[8];
         merge_raw<DTYPE, HAS_U, HAS_T>(raw, s2, t2, y);
         const float m8 = max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]);
-        atomicAdd(&sm.hist[float_key(canonical(m8)) >> 21], 1u);
+        if (cfg.sample_all) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) atomicAdd(&sm.hist[float_key(canonical(y[k])) >> 21], 1u);
+        } else {
+          atomicAdd(&sm.hist[float_key(canonical(m8)) >> 21], 1u);
+        }
         smax = fmaxf(smax, m8);
       }
     }
@@ -195,7 +201,8 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
       if (tid == 0) *abort_flag = 1;
       continue;
     }
-    // at least m group maxima, hence at least m sample elements, are >= the lower edge of this bin
+    // at least m group maxima (or, binning everything, m elements), hence at least m sample elements, are >=
+    // the lower edge of this bin
     find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kRcFBin);
     const int cbin = sm.ctl[kRcFBin];
     float floor_y = cbin >= 0 ? key_float((uint32_t)cbin << 21) : lowest;
@@ -504,7 +511,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       // that the bins (= st_ids) stay clear
       group_sync<NT_P, BAR_P>();
       if (tid == 0) mbar_arrive(sm.cand_free);
-      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals));
+      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals), kRowStatusRedone);
       continue;
     }
     // linear bins over [tau0, vmax]; monotone in y, so a higher bin never holds a smaller value
@@ -604,7 +611,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       // the threshold bin was too crowded for the on-chip ranking: exact any-shape path from global memory.
       // The bins were cleared when they were read; the any-shape path's scratch sits on st_vals.
       for (int j = tid; j < kSelBins; j += NT_P) sm.sel[j] = 0;
-      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals));
+      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals), kRowStatusRedone);
       continue;
     }
     // ---- normalise, write the row, draw from it ----

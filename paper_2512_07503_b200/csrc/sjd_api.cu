@@ -51,11 +51,22 @@ constexpr size_t kSmemLimit = 227u * 1024u;
 
 // Decide whether the single-pass pipelined kernel can take this shape, and with which sampling
 // parameters.  The sample is every SS-th 256-element tile of a row; its rank-m value (from the top)
-// becomes the candidate threshold.  m is chosen 3.5 standard deviations above K/SS, so that a row with
-// exchangeable entries fails to deliver K candidates with probability below 3e-4 (such a row is redone
-// by the any-shape path, never answered wrongly).  The on-chip lists must hold the expected number of
+// becomes the candidate threshold.  m is chosen 4.5 standard deviations above K/SS (sample_rank), so that
+// a row with exchangeable entries almost never fails to deliver K candidates (such a row is redone by the
+// any-shape path, never answered wrongly).  The on-chip lists must hold the expected number of
 // candidates with a margin: four standard deviations for the row's total, and for the share of one
 // filter thread (a Poisson count) a tail below 1e-6.
+// Rank m of the sample element that serves as the first threshold, for an expected a = kcap / S of the row's
+// kcap largest inside a sample of one S-th of the row.  The number of those that really fall in the sample
+// is at most Poisson(a)-distributed (drawing without replacement only narrows it), so m = a + z sqrt(m),
+// i.e. sqrt(m) = z/2 + sqrt(z^2/4 + a), leaves the threshold above the true one (too few candidates, the
+// row redone by the any-shape path at many times the cost) with a probability below 4e-6 per row at z = 4.5.
+int sample_rank(double a) {
+  constexpr double z = 4.5;
+  const double root = z / 2 + std::sqrt(z * z / 4 + a);
+  return (int)std::ceil(root * root);
+}
+
 bool plan_pipeline(const sjd_params* P, int kcap, sjd::PipeCfg* cfg, size_t* smem) {
   const int V = P->V;
   if (kcap > sjd::kKcapMax || V % sjd::kTileElems != 0) return false;
@@ -80,8 +91,7 @@ bool plan_pipeline(const sjd_params* P, int kcap, sjd::PipeCfg* cfg, size_t* sme
     if (ns > kMaxStages) ns = kMaxStages;
     const int n_sample = V / ss;
     const double a = (double)kcap / ss;
-    const double root = 1.75 + std::sqrt(1.75 * 1.75 + a);
-    const int m = (int)std::ceil(root * root);
+    const int m = sample_rank(a);
     if (m > n_sample / 2 || m > 32 * sample_tiles) continue;  // the rank must exist among the group maxima too
     const double mean = (double)m * ss, sd = (double)ss * std::sqrt((double)m);
     if (mean + 4.0 * sd > (double)sjd::kDenseCap) continue;
@@ -118,7 +128,7 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 // Same sampling rule as plan_pipeline; the sample is stage 0, i.e. 1/S of the row.
-bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem) {
+bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem, bool need_encoder = true) {
   const int V = P->V;
   const int es = P->logits_dtype == SJD_BF16 ? 2 : 4;
   const int bw = 64 / es;  // elements per stage and range
@@ -134,15 +144,18 @@ bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem
   if (mask_words > sjd::kMaskWordsMax) return false;
   const int n_sample = sjd::kRangeThreads * bw;
   const double a = (double)kcap / S;
-  const double root = 1.75 + std::sqrt(1.75 * 1.75 + a);
-  const int m = (int)std::ceil(root * root);
-  if (m > n_sample / 2 || m > n_sample / 8) return false;  // the rank must exist among the group maxima too
+  const int m = sample_rank(a);
+  if (m > n_sample / 2) return false;
+  const int sample_all = m > n_sample / 8 ? 1 : 0;  // the rank must exist among what the first pass bins
   const double mean = (double)m * S, sd = (double)S * std::sqrt((double)m);
   if (mean + 4.0 * sd > (double)sjd::kRangeDenseCap) return false;
-  const double per_thread = (mean * (S - 1) / S + 2.1 * m) / sjd::kRangeThreads;  // pair entries, sample kept against a floor
+  // pair entries: the candidates outside the sample, and the sample kept against a floor below its rank-m
+  // element (the floor from group maxima lies lower than the one from every element)
+  const double per_thread = (mean * (S - 1) / S + (sample_all ? 1.7 : 2.1) * m) / sjd::kRangeThreads;
   if (per_thread + 5.0 * std::sqrt(per_thread) + 1.0 > (double)(sjd::kListCap - 4)) return false;
-  if (encode_tiled_fn() == nullptr) return false;
+  if (need_encoder && encode_tiled_fn() == nullptr) return false;
   cfg->sample_rank = m;
+  cfg->sample_all = sample_all;
   cfg->stages = S;
   cfg->range_len = R;
   cfg->mask_words = mask_words;
@@ -418,6 +431,24 @@ int fill_advance(sjd::AdvanceArgs* a, const sjd_params* P, int32_t n_total, uint
 }  // namespace
 
 extern "C" {
+
+int sjd_row_kernel(const sjd_params* P) {
+  if (!P) return SJD_ERR_NULL;
+  if (P->struct_size != (int32_t)sizeof(sjd_params)) return SJD_ERR_STRUCT;
+  if (P->B < 0 || P->W < 1 || P->W > SJD_W_MAX || P->V < 8 || (P->V % 8) != 0 || P->top_k < 1) return SJD_ERR_SHAPE;
+  if (P->logits_dtype != SJD_F32 && P->logits_dtype != SJD_BF16) return SJD_ERR_DTYPE;
+  const int64_t esize = P->logits_dtype == SJD_BF16 ? 2 : 4;
+  if ((P->stride_b * esize) % 16 != 0 || (P->stride_w * esize) % 16 != 0 || P->stride_w < P->V || P->stride_b < 0)
+    return SJD_ERR_ALIGN;
+  const int kcap = P->top_k < P->V ? P->top_k : P->V;
+  sjd::PipeCfg cfg;
+  sjd::RangeCfg rcfg;
+  size_t smem = 0;
+  const bool fast = !(P->flags & (SJD_FLAG_FORCE_GENERIC | SJD_FLAG_FORCE_TILES));
+  if (fast && plan_ranges(P, kcap, &rcfg, &smem, false)) return SJD_ROWS_RANGES;
+  if (!(P->flags & SJD_FLAG_FORCE_GENERIC) && plan_pipeline(P, kcap, &cfg, &smem)) return SJD_ROWS_TILES;
+  return SJD_ROWS_GENERIC;
+}
 
 int sjd_window_init(const sjd_params* P, int32_t n_total, uint64_t philox_seed, int32_t* win_len, int32_t* pos_base,
                     int32_t* iteration, int32_t* drafts, sjd_probs* draft_probs) {

@@ -14,7 +14,7 @@ constexpr int kFlagDraftAll = 2;
 constexpr int kQUniform = -1;
 
 constexpr int kOutInvalid = 0, kOutAccepted = 1, kOutResidual = 2, kOutReused = 3, kOutResampled = 4;
-constexpr int kStatusQtok = 1, kStatusEmptyResidual = 2, kStatusDegenerate = 4, kStatusTimeout = 8;
+constexpr int kStatusQtok = 1, kStatusEmptyResidual = 2, kStatusDegenerate = 4, kStatusTimeout = 8, kStatusRedone = 16;
 
 struct VerifyArgs {
   int B, W, V, kcap;
@@ -101,6 +101,7 @@ __device__ void verify_sequence(const VerifyArgs& a, int b, int tid, VerifySmem&
     const RowScratch rs = a.scratch[base + i];
     int st = (rs.status & kRowStatusDegenerate) ? kStatusDegenerate : 0;
     if (rs.status & kRowStatusTimeout) st |= kStatusTimeout;
+    if (rs.status & kRowStatusRedone) st |= kStatusRedone;
     if (!draft_all) {
       const float q = a.q_tok[base + i];
       const float ratio = likelihood_ratio(rs.p_tok, q);

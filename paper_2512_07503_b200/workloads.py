@@ -68,6 +68,30 @@ CONFIGS = {
 }
 
 
+def _sweep():
+    """Wider shapes around the headline configuration, same recipe: the window sizes of the paper's window
+    ablation (16 to 512), the top-K values of its sampling ablation, and the vocabularies of the models it
+    accelerates (16,384, 32,768 and 65,536 entries).  Batches keep the row count near the headline's 1,024."""
+    base = CONFIGS["cfg4"]
+    out = {}
+    for W, B in ((16, 64), (32, 32), (96, 11), (250, 4), (512, 2)):
+        out[f"w{W}"] = base.scaled(name=f"w{W}", B=B, W=W, seed=100 + W)
+    for K in (1, 10, 100, 500, 1000, 8192):
+        out[f"k{K}"] = base.scaled(name=f"k{K}", top_k=K, seed=200 + K % 97)
+    out["v32k"] = base.scaled(name="v32k", V=32768, seed=301)
+    out["v16k"] = base.scaled(name="v16k", V=16384, seed=302)
+    out["v16k_f32"] = base.scaled(name="v16k_f32", V=16384, dtype=F32, seed=303)
+    return out
+
+
+SWEEP = _sweep()
+
+
+def workload(name: str) -> Workload:
+    """A benchmark configuration or a sweep shape by name."""
+    return CONFIGS[name] if name in CONFIGS else SWEEP[name]
+
+
 def to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round fp32 to bf16 (nearest, ties to even) and return the uint16 patterns."""
     b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)

@@ -101,6 +101,7 @@ def check_parity(cond, uncond, drafts, qprobs, kw, win_len, *, expect_flagged_be
     rep = compare.compare_step(got.accept_len, got.tokens, got.tok_prob, got.flags, got.ids, got.vals, got.cnt, ref,
                                drafts, win_len, kw["flags"])
     assert rep.ok(), rep.summary() + "\n" + "\n".join(rep.errors)
-    assert np.array_equal(got.status, ref.status), (got.status, ref.status)
+    # bit 16 only says that a row took the any-shape path inside the library: no counterpart in the oracle
+    assert np.array_equal(got.status & ~16, ref.status), (got.status, ref.status)
     assert rep.flagged <= max(2, expect_flagged_below * rep.positions), rep.summary()
     return rep, got, ref

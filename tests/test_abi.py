@@ -52,3 +52,24 @@ def test_params_struct_matches_header_layout():
         for part in decl.split(","):
             fields.append(re.findall(r"([A-Za-z_][A-Za-z0-9_]*)\s*$", part.strip())[0])
     assert fields == [f for f, _ in sjd.sjd_params._fields_]
+
+
+def test_row_kernel_query_needs_no_gpu_and_follows_the_shape_rules():
+    import ctypes as C
+    from paper_2512_07503_b200 import binding as B
+
+    def params(V, top_k, dtype=B.SJD_BF16, flags=0, W=8):
+        p = B.sjd_params()
+        p.struct_size = C.sizeof(B.sjd_params)
+        p.B, p.W, p.V, p.logits_dtype, p.top_k, p.flags = 2, W, V, dtype, top_k, flags
+        p.stride_b, p.stride_w = W * V, V
+        return p
+
+    assert B.sjd_row_kernel(params(65536, 2000)) == B.SJD_ROWS_RANGES
+    assert B.sjd_row_kernel(params(65536, 1000, flags=B.SJD_FLAG_FORCE_TILES)) == B.SJD_ROWS_TILES
+    assert B.sjd_row_kernel(params(65536, 2000, flags=B.SJD_FLAG_FORCE_GENERIC)) == B.SJD_ROWS_GENERIC
+    assert B.sjd_row_kernel(params(65536, 8192)) == B.SJD_ROWS_GENERIC      # kcap above what the on-chip path stages
+    assert B.sjd_row_kernel(params(1032, 7, dtype=B.SJD_F32)) == B.SJD_ROWS_GENERIC
+    import pytest
+    with pytest.raises(B.SjdError):
+        B.sjd_row_kernel(params(65530, 10))

@@ -171,6 +171,7 @@ def test_pipeline_all_equal_logits_overflow_the_candidate_lists():
     drafts = np.array([[3, 70, 4000]], np.int32)
     rep, got, ref = check_parity(inp.cond, inp.uncond, drafts, q, step_kwargs(inp), inp.win_len)
     assert np.array_equal(got.ids[0, 0], np.arange(64))
+    assert got.status[0] & 16          # SJD_STATUS_ROW_REDONE: the rows went through the any-shape path
 
 
 def test_pipeline_bf16_ties_at_the_threshold():
@@ -199,18 +200,53 @@ def test_pipeline_structured_row_defeats_the_sample():
         inp.cond[:, :, t * 256:(t + 1) * 256] -= 50.0
         inp.uncond[:, :, t * 256:(t + 1) * 256] -= 50.0
     prev = oracle_prime(inp)
-    check_parity(inp.cond, inp.uncond, prev.tokens, prev.probs, step_kwargs(inp), inp.win_len)
+    rep, got, ref = check_parity(inp.cond, inp.uncond, prev.tokens, prev.probs, step_kwargs(inp, flags=oracle.FLAG_REUSE | 8),
+                                 inp.win_len)
+    assert got.status[0] & 16
     # and the opposite: the sample tiles hold the largest values, so the threshold is too high
     inp2 = wk.make_step_inputs(wl)
     for t in range(0, 32, 8):
         inp2.cond[:, :, t * 256:(t + 1) * 256] += 50.0
         inp2.uncond[:, :, t * 256:(t + 1) * 256] += 50.0
     prev2 = oracle_prime(inp2)
-    check_parity(inp2.cond, inp2.uncond, prev2.tokens, prev2.probs, step_kwargs(inp2), inp2.win_len)
+    rep, got, ref = check_parity(inp2.cond, inp2.uncond, prev2.tokens, prev2.probs,
+                                 step_kwargs(inp2, flags=oracle.FLAG_REUSE | 8), inp2.win_len)
+    assert got.status[0] & 16
+
+
+@pytest.mark.parametrize("dtype,V,K", [(wk.BF16, 16384, 500), (wk.F32, 16384, 300), (wk.BF16, 16384, 2000)])
+def test_range_kernel_structured_row_defeats_the_sample(dtype, V, K):
+    # the range kernel samples the first 64 bytes of each of the 256 id ranges of a row: make exactly those
+    # entries very small (threshold far too low, lists overflow) or very large (too few candidates); both
+    # ways the row is redone by the any-shape path and stays exact
+    from gpu_harness import check_parity, oracle_prime, step_kwargs
+    wl = wk.CONFIGS["cfg2"].scaled(B=1, W=3, V=V, top_k=K, dtype=dtype)
+    R, bw = V // 256, 64 // (2 if dtype == wk.BF16 else 4)
+    sample = (np.arange(V) % R) < bw
+    for shift in (-50.0, 50.0):
+        inp = wk.make_step_inputs(wl)
+        for arr in (inp.cond, inp.uncond):
+            if dtype == wk.BF16:
+                f = wk.bf16_bits_to_f32(arr)
+                f[:, :, sample] += np.float32(shift)
+                arr[:] = wk.to_bf16_bits(f)
+            else:
+                arr[:, :, sample] += np.float32(shift)
+        prev = oracle_prime(inp)
+        rep, got, ref = check_parity(inp.cond, inp.uncond, prev.tokens, prev.probs, step_kwargs(inp), inp.win_len)
+        assert got.status[0] & 16, shift
+
+
+def test_ordinary_rows_are_not_redone():
+    rep, got, ref, inp, prev = _run(wk.CONFIGS["cfg2"].scaled(W=8))
+    assert not (got.status[0] & 16)
+    rep, got, ref, inp, prev = _run(wk.SWEEP["v16k"].scaled(B=2, W=8))
+    assert not np.any(got.status & 16)
 
 
 @pytest.mark.parametrize("force", [4, 8])  # SJD_FLAG_FORCE_GENERIC, SJD_FLAG_FORCE_TILES
 def test_every_row_kernel_gives_the_same_answer(force):
     # the same shapes through the any-shape kernel and the tile-dealing kernel instead of the range kernel
     _run(wk.CONFIGS["cfg2"].scaled(W=6), flags=oracle.FLAG_REUSE | force)
+    _run(wk.CONFIGS["cfg2"].scaled(W=6, top_k=1000), flags=oracle.FLAG_REUSE | force)   # a shape the tile kernel takes
     _run(wk.CONFIGS["cfg3"].scaled(B=6), flags=oracle.FLAG_REUSE | force)
