@@ -21,6 +21,12 @@ constexpr int kRowStatusRedone = 4;   // the single-pass kernel handed the row t
 // Philox4x32-10 (Salmon et al., SC'11): counter = (position, sequence, iteration, purpose),
 // key = (seed low, seed high).
 // ------------------------------------------------------------------------------------------------
+// Programmatic dependent launch: a kernel lets the next kernel of its stream be scheduled early
+// (allow_dependent_launch), and that kernel blocks in grid_dependency_wait() until the first has completed
+// and its memory operations are visible.
+__device__ __forceinline__ void allow_dependent_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 struct Philox4 {
   uint32_t x0, x1, x2, x3;
 };

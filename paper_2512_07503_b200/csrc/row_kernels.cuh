@@ -198,7 +198,12 @@ template <int DTYPE, int NT>
 __global__ void __launch_bounds__(NT) rows_generic_kernel(const RowArgs a) {
   __shared__ GenericSmem sm;
   const int rows = a.B * a.W;
-  for (int row = blockIdx.x; row < rows; row += gridDim.x) row_generic<DTYPE, NT, 0>(a, row, threadIdx.x, sm);
+  grid_dependency_wait();  // a launch allowed to overlap the stream's previous kernel waits for its end here
+  for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    // from the block's last row on, the verification grid may be scheduled (it waits for this grid's end)
+    if (row + (int)gridDim.x >= rows) allow_dependent_launch();
+    row_generic<DTYPE, NT, 0>(a, row, threadIdx.x, sm);
+  }
 }
 
 }  // namespace sjd

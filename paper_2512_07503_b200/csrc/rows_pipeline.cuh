@@ -407,6 +407,8 @@ __device__ __forceinline__ void filter_role(const RowArgs& a, const PipeCfg& cfg
   uint32_t n_row = 0;
   bool dead = false;
   for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    // from the block's last row on, the verification grid may be scheduled (it waits for this grid's end)
+    if (row + (int)gridDim.x >= rows) allow_dependent_launch();
     const int b = row / a.W, i = row - b * a.W;
     const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
     if (i >= L || dead) continue;
@@ -613,6 +615,8 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
         if (it < kItersMax) sm.tile_of[warp * kItersMax + it++] = (uint16_t)sched.global_tile(s, j, TPS);
     }
   }
+  // only shared memory so far; a launch allowed to overlap the stream's previous kernel waits for its end here
+  grid_dependency_wait();
   __syncthreads();
 
   volatile int* abort_flag = sm.ctl + kCtlAbort;
@@ -702,6 +706,8 @@ __global__ void __launch_bounds__((NF + NP + 1) * 32, 1) rows_pipeline_kernel(co
   uint32_t n_row = 0;
   bool dead = false;
   for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    // from the block's last row on, the verification grid may be scheduled (it waits for this grid's end)
+    if (row + (int)gridDim.x >= rows) allow_dependent_launch();
     const int b = row / a.W, i = row - b * a.W;
     const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
     RowScratch* rs = a.scratch + row;

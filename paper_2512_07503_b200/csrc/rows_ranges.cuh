@@ -168,6 +168,8 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
   };
 
   for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    // from the block's last row on, the verification grid may be scheduled (it waits for this grid's end)
+    if (row + (int)gridDim.x >= rows) allow_dependent_launch();
     const int b = row / a.W, i = row - b * a.W;
     const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
     if (i >= L || dead) continue;
@@ -409,6 +411,9 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   }
   for (int j = threadIdx.x; j < kHistBins; j += blockDim.x) sm.hist[j] = 0;
   for (int j = threadIdx.x; j < kSelBins; j += blockDim.x) sm.sel[j] = 0;
+  // everything above touched shared memory only; global memory is read and written from here on, so a
+  // launch that was allowed to overlap the previous kernel of the stream waits for that kernel's end here
+  grid_dependency_wait();
   __syncthreads();
   volatile int* abort_flag = sm.ctl + kRcAbort;
 
@@ -474,6 +479,8 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   uint32_t n_row = 0;
   bool dead = false;
   for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    // from the block's last row on, the verification grid may be scheduled (it waits for this grid's end)
+    if (row + (int)gridDim.x >= rows) allow_dependent_launch();
     const int b = row / a.W, i = row - b * a.W;
     const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
     RowScratch* rs = a.scratch + row;

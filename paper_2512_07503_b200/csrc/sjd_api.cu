@@ -177,6 +177,26 @@ bool make_range_map(CUtensorMap* map, const void* base, const sjd_params* P, con
   return r == CUDA_SUCCESS;
 }
 
+// Launch as a programmatic dependent of the stream's previous kernel: when that kernel allows it (ours do
+// near their end), this grid's blocks are placed and set up early and wait inside the kernel
+// (grid_dependency_wait) until the previous kernel has completed.  After a kernel that does not take part,
+// an event or a copy this is an ordinary launch.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool dependent,
+                         Args&&... args) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid;
+  lc.blockDim = block;
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&lc, kern, std::forward<Args>(args)...);
+}
+
 template <int DTYPE>
 cudaError_t launch_ranges(const sjd::RowArgs& ra, const sjd::RangeCfg& cfg, const CUtensorMap& mc, const CUtensorMap& mu,
                           size_t smem, int grid, cudaStream_t st) {
@@ -187,8 +207,7 @@ cudaError_t launch_ranges(const sjd::RowArgs& ra, const sjd::RangeCfg& cfg, cons
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<grid, (8 + kFinisherWarps + 1) * 32, smem, st>>>(ra, cfg, mc, mu);
-  return cudaGetLastError();
+  return launch_after(kern, dim3((unsigned)grid), dim3((8 + kFinisherWarps + 1) * 32), smem, st, true, ra, cfg, mc, mu);
 }
 
 template <int DTYPE>
@@ -200,8 +219,7 @@ cudaError_t launch_pipeline(const sjd::RowArgs& ra, const sjd::PipeCfg& cfg, siz
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<grid, (kFilterWarps + kFinisherWarps + 1) * 32, smem, st>>>(ra, cfg);
-  return cudaGetLastError();
+  return launch_after(kern, dim3((unsigned)grid), dim3((kFilterWarps + kFinisherWarps + 1) * 32), smem, st, true, ra, cfg);
 }
 
 // Scratch of sjd_step_static(): lives in the library's device image, so every GPU that loads the library
@@ -339,11 +357,9 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
                                       : launch_pipeline<0>(ra, cfg, smem, grid, stream);
     } else {
       const int grid = rows < 4 * sm_count() ? rows : 4 * sm_count();
-      if (P->logits_dtype == SJD_BF16)
-        sjd::rows_generic_kernel<1, kGenericThreads><<<grid, kGenericThreads, 0, stream>>>(ra);
-      else
-        sjd::rows_generic_kernel<0, kGenericThreads><<<grid, kGenericThreads, 0, stream>>>(ra);
-      e = cudaGetLastError();
+      e = P->logits_dtype == SJD_BF16
+              ? launch_after(sjd::rows_generic_kernel<1, kGenericThreads>, dim3((unsigned)grid), dim3(kGenericThreads), 0, stream, true, ra)
+              : launch_after(sjd::rows_generic_kernel<0, kGenericThreads>, dim3((unsigned)grid), dim3(kGenericThreads), 0, stream, true, ra);
     }
     if (e != cudaSuccess) return cuda_fail(e, "row kernel launch");
     ++g_launches;
@@ -378,8 +394,11 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
   va.out_flags = P->out_flags;
   va.status = P->status;
   {
-    sjd::verify_kernel<kVerifyThreads><<<P->B, kVerifyThreads, 0, stream>>>(va);
-    const cudaError_t e = cudaGetLastError();
+    // directly behind the row kernel the verification grid is launched as its programmatic dependent: its
+    // blocks are placed as the row kernel's last blocks retire and wait inside the kernel for its completion.
+    // An event recorded in between makes it an ordinary launch.
+    const cudaError_t e = launch_after(sjd::verify_kernel<kVerifyThreads>, dim3((unsigned)P->B), dim3(kVerifyThreads), 0, stream,
+                                       P->ev_rows_end == nullptr, va);
     if (e != cudaSuccess) return cuda_fail(e, "verify kernel launch");
     ++g_launches;
   }

@@ -224,6 +224,12 @@ __device__ void verify_sequence(const VerifyArgs& a, int b, int tid, VerifySmem&
 template <int NT>
 __global__ void __launch_bounds__(NT) verify_kernel(const VerifyArgs a) {
   __shared__ VerifySmem sm;
+  // Launched with programmatic stream serialisation right behind the row kernel: the grid may be scheduled
+  // while that kernel's last rows are still running, and waits here until all of its writes are visible.
+  // A no-op after an ordinary launch.
+  grid_dependency_wait();
+  // a following kernel that waits the same way (the next step's row kernel) may set itself up meanwhile
+  allow_dependent_launch();
   for (int b = blockIdx.x; b < a.B; b += gridDim.x) verify_sequence<NT, 0>(a, b, threadIdx.x, sm);
 }
 
