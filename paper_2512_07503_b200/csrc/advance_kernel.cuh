@@ -56,6 +56,10 @@ __device__ __forceinline__ int random_token(int pos, int seq, int iter, int V, u
 // One block per (sequence, next-window row).
 template <int NT>
 __global__ void __launch_bounds__(NT) advance_rows_kernel(const AdvanceArgs a) {
+  // launched as a programmatic dependent of the step's verification kernel: wait for its results, then
+  // let the kernel behind this one be placed early in turn
+  grid_dependency_wait();
+  allow_dependent_launch();
   const int b = blockIdx.x / a.W, i = blockIdx.x - b * a.W;
   const int L = min(max(a.win_len[b], 0), a.W);
   const int pos0 = a.pos_base[b];
@@ -157,6 +161,8 @@ __global__ void __launch_bounds__(NT) advance_rows_kernel(const AdvanceArgs a) {
 
 // One thread per sequence: the window state after the commit.  Runs after advance_rows_kernel.
 __global__ void advance_state_kernel(const AdvanceArgs a) {
+  grid_dependency_wait();  // advance_rows_kernel reads the state this kernel overwrites
+  allow_dependent_launch();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= a.B) return;
   const int L = min(max(a.win_len[b], 0), a.W);

@@ -499,12 +499,10 @@ int sjd_window_advance(const sjd_params* P, int32_t n_total, uint64_t philox_see
   a.committed = committed;
   a.n_committed = n_committed;
   cudaStream_t st = static_cast<cudaStream_t>(P->stream);
-  sjd::advance_rows_kernel<256><<<P->B * P->W, 256, 0, st>>>(a);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_after(sjd::advance_rows_kernel<256>, dim3((unsigned)(P->B * P->W)), dim3(256), 0, st, true, a);
   if (e != cudaSuccess) return cuda_fail(e, "window advance launch");
   ++g_launches;
-  sjd::advance_state_kernel<<<(P->B + 127) / 128, 128, 0, st>>>(a);
-  e = cudaGetLastError();
+  e = launch_after(sjd::advance_state_kernel, dim3((unsigned)((P->B + 127) / 128)), dim3(128), 0, st, true, a);
   if (e != cudaSuccess) return cuda_fail(e, "window state launch");
   ++g_launches;
   return SJD_OK;

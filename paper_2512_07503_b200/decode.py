@@ -1,6 +1,11 @@
 """Decode loop on the device: sjd_step + sjd_window_advance per Jacobi iteration, with every buffer
 allocated once.  The model's forward pass is a callable that maps the current window to cond / uncond
-logits on the device.  Marshalling only: all arithmetic runs in the library's kernels."""
+logits on the device.  Marshalling only: all arithmetic runs in the library's kernels.
+
+With ``use_graphs=True`` the four kernels of an iteration are captured once per buffer parity into a CUDA
+graph and replayed, which removes the host's launch work from the critical path of small windows; the
+logits then have to sit in the loop's own buffers (``cond_buf`` / ``uncond_buf``; other tensors are copied
+there)."""
 from __future__ import annotations
 
 from typing import Callable, Optional, Tuple
@@ -14,7 +19,7 @@ class DecodeLoop:
     def __init__(self, *, batch: int, window: int, vocab: int, n_total: int, logits_dtype: torch.dtype, top_k: int,
                  cfg_scale: float = 1.0, inv_temperature: float = 1.0, reuse_tau: float = 0.5, reuse: bool = True,
                  seed: int = 0, seq_base: int = 0, init_mode: int = B.SJD_INIT_RANDOM, grid_width: int = 1,
-                 device="cuda:0"):
+                 use_graphs: bool = False, guidance: bool = True, device="cuda:0"):
         self.B, self.W, self.V, self.N = batch, window, vocab, n_total
         self.kcap = min(top_k, vocab)
         self.seed, self.device = seed, torch.device(device)
@@ -38,6 +43,12 @@ class DecodeLoop:
                                     pos_base=self.pos_base, iteration=self.iteration, status=self.status,
                                     seq_base=seq_base, init_mode=init_mode, grid_width=grid_width)
         del proto
+        self.use_graphs = use_graphs
+        self.graphs = [None, None]   # one per buffer parity
+        self.eager_done = [False, False]
+        if use_graphs:
+            self.cond_buf = torch.empty(batch, window, vocab, dtype=logits_dtype, device=dev)
+            self.uncond_buf = torch.empty_like(self.cond_buf) if guidance else None
         self.ws = torch.empty(B.sjd_workspace_bytes(self.params), dtype=torch.uint8, device=dev)
         self.params.workspace, self.params.workspace_bytes = self.ws.data_ptr(), self.ws.numel()
         B.sjd_window_init(self.params, n_total, seed, self.win_len, self.pos_base, self.iteration, self.drafts[0], self.q[0])
@@ -47,15 +58,39 @@ class DecodeLoop:
     def window_tokens(self) -> torch.Tensor:
         return self.drafts[self.cur]
 
-    def step(self, cond: torch.Tensor, uncond: Optional[torch.Tensor]) -> None:
-        """One Jacobi iteration on logits [B,W,V] for the current window (asynchronous)."""
-        c, n = self.cur, self.cur ^ 1
+    def _launch(self, cond, uncond, c: int) -> None:
+        n = c ^ 1
         p = self.params
         p.stride_b, p.stride_w = cond.stride(0), cond.stride(1)
+        p.stream = torch.cuda.current_stream(self.device).cuda_stream
         B.sjd_step(cond, uncond, self.drafts[c], self.q[c], p, self.seed, self.acc, self.toks, self.out)
         B.sjd_window_advance(p, self.N, self.seed, self.acc, self.toks, self.out, self.win_len, self.pos_base,
                              self.iteration, self.drafts[n], self.q[n], self.committed, self.n_committed)
-        self.cur = n
+
+    def step(self, cond: torch.Tensor, uncond: Optional[torch.Tensor]) -> None:
+        """One Jacobi iteration on logits [B,W,V] for the current window (asynchronous)."""
+        c = self.cur
+        if not self.use_graphs:
+            self._launch(cond, uncond, c)
+        else:
+            if (uncond is None) != (self.uncond_buf is None):
+                raise B.SjdError("guidance must match the loop's `guidance` setting when graphs are used")
+            if cond.data_ptr() != self.cond_buf.data_ptr():
+                self.cond_buf.copy_(cond)
+            if uncond is not None and uncond.data_ptr() != self.uncond_buf.data_ptr():
+                self.uncond_buf.copy_(uncond)
+            if not self.eager_done[c]:
+                # first use of this parity: an ordinary launch (it also performs the one-time kernel set-up)
+                self._launch(self.cond_buf, self.uncond_buf, c)
+                self.eager_done[c] = True
+            else:
+                if self.graphs[c] is None:
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g):
+                        self._launch(self.cond_buf, self.uncond_buf, c)
+                    self.graphs[c] = g
+                self.graphs[c].replay()
+        self.cur = c ^ 1
         self.steps += 1
 
     def done(self) -> bool:

@@ -13,7 +13,8 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64, init_mode=0, grid_width=1, windows=False):
+def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64, init_mode=0, grid_width=1, windows=False,
+          use_graphs=False):
     from paper_2512_07503_b200.decode import DecodeLoop
     src = wk.MarkovSource(V, N, dtype, states=states)
     flags = oracle.FLAG_REUSE if reuse else 0
@@ -25,7 +26,7 @@ def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64, init_mode=0,
 
     tdt = torch.bfloat16 if dtype == wk.BF16 else torch.float32
     dl = DecodeLoop(batch=B, window=W, vocab=V, n_total=N, logits_dtype=tdt, top_k=top_k, cfg_scale=3.0, reuse=reuse,
-                    seed=seed, init_mode=init_mode, grid_width=grid_width, device=DEV)
+                    seed=seed, init_mode=init_mode, grid_width=grid_width, use_graphs=use_graphs, device=DEV)
 
     def up(a):
         if dtype == wk.BF16:
@@ -71,6 +72,14 @@ def test_spatial_prior_initialisation_matches_the_oracle(B, W, V, N, K, dtype, G
     assert got[1] == ref[1], (got[1], ref[1])
     assert np.array_equal(got[2], ref[2])
     assert np.array_equal(got[0], ref[0])
+
+
+@pytest.mark.parametrize("mode", [0, 4])
+def test_graph_replay_gives_the_same_trajectory(mode):
+    # every iteration after the first two replays a captured CUDA graph of the four kernels
+    got, ref = _both(2, 12, 8192, 70, 300, wk.BF16, init_mode=mode, grid_width=16, windows=True, use_graphs=True)
+    assert got[1] == ref[1] and np.array_equal(got[2], ref[2]) and np.array_equal(got[0], ref[0])
+    assert got[1] > 6
 
 
 def test_random_initialisation_windows_match_the_oracle():
