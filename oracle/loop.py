@@ -21,10 +21,10 @@ strategies and fixes nothing else; the choices below are this implementation's):
   * "repeat left" copies the token of p-1, "repeat above" the token of p-G (of p-1 when p < G); the draft
     is deterministic, so its reference distribution is the point mass on that token (one entry of
     probability 1), which keeps the accept test and the residual exact;
-  * "sample left" / "sample above" draw from a sparse distribution the step just produced: the last window
-    row's for "left" (p-1 when p is the first new slot; later new slots have no prediction of their own and
-    use the same row), the row of position p-G for "above", stepping a further G back while that position
-    is itself a new slot; the draw is the fixed-point inverse CDF on one Philox block (purpose 5) and the
+  * "sample left" / "sample above" draw from a sparse distribution the step just produced: for "left" the
+    one predicted for position p-1, or the last window row's when p-1 lies behind the verified window (with
+    refinement every new slot does); for "above" the row of position p-G, stepping a further G back while
+    that position lies behind the verified window; the draw is the fixed-point inverse CDF on one Philox block (purpose 5) and the
     reference distribution is the one drawn from.  When position p-G was verified before this step, its
     distribution no longer exists and the slot falls back to "repeat above"; when p < G it falls back to
     "sample left";
@@ -108,8 +108,9 @@ def window_init(B, W, V, kcap, n_total, seed, seq_base=0, iteration0=0, init_mod
 
 
 def window_advance(w: Window, accept_len, step_tokens, step_probs: Probs, V, n_total, seed, seq_base=0,
-                   init_mode=INIT_RANDOM, grid_width=0):
-    """Commit, shift and refill.  Returns (next window, committed counts)."""
+                   init_mode=INIT_RANDOM, grid_width=0, refine=True):
+    """Commit, shift and refill.  Returns (next window, committed counts).  With refine=False (the paper's
+    "no refinement" ablation) nothing is shifted: every slot behind the committed tokens is newly initialised."""
     B, W = w.drafts.shape
     kcap = w.probs.ids.shape[-1]
     nxt = Window(np.full((B, W), -1, np.int32), Probs.empty(B, W, kcap), np.zeros(B, np.int32), np.zeros(B, np.int32),
@@ -125,7 +126,7 @@ def window_advance(w: Window, accept_len, step_tokens, step_probs: Probs, V, n_t
         nxt.pos_base[b], nxt.win_len[b] = p1, L1
         for i in range(L1):
             src = i + c
-            if src < L:
+            if refine and src < L:
                 nxt.drafts[b, i] = step_tokens[b, src]
                 nxt.probs.tok_prob[b, i] = step_probs.tok_prob[b, src]
                 n = int(step_probs.cnt[b, src])
@@ -139,11 +140,13 @@ def window_advance(w: Window, accept_len, step_tokens, step_probs: Probs, V, n_t
                 _set_uniform(nxt.probs, b, i, V)
                 continue
 
+            known = L if refine else c        # window rows whose token survives into the next iteration
+
             def token_at(r):
                 # r < p; new slots before p are already filled in nxt
                 if r < p0:
                     return int(w.committed[b, r])
-                if r < p0 + L:
+                if r < p0 + known:
                     return int(step_tokens[b, r - p0])
                 return int(nxt.drafts[b, r - p1])
 
@@ -153,7 +156,8 @@ def window_advance(w: Window, accept_len, step_tokens, step_probs: Probs, V, n_t
                 nxt.drafts[b, i] = token_at(p - grid_width if above else p - 1)
                 _set_point_mass(nxt.probs, b, i, nxt.drafts[b, i])
             elif not above:
-                nxt.drafts[b, i] = _draw_from_row(nxt.probs, b, i, step_probs, b, L - 1, seed, p, seq_base + b, it)
+                left = min(p - 1 - p0, L - 1)   # the prediction made for position p-1, else the last one made
+                nxt.drafts[b, i] = _draw_from_row(nxt.probs, b, i, step_probs, b, left, seed, p, seq_base + b, it)
             else:
                 r = p - grid_width
                 while r >= p0 + L:
@@ -164,13 +168,14 @@ def window_advance(w: Window, accept_len, step_tokens, step_probs: Probs, V, n_t
                     nxt.drafts[b, i] = int(w.committed[b, r])
                     _set_point_mass(nxt.probs, b, i, nxt.drafts[b, i])
                 else:
-                    nxt.drafts[b, i] = _draw_from_row(nxt.probs, b, i, step_probs, b, L - 1, seed, p, seq_base + b, it)
+                    left = min(p - 1 - p0, L - 1)
+                    nxt.drafts[b, i] = _draw_from_row(nxt.probs, b, i, step_probs, b, left, seed, p, seq_base + b, it)
     return nxt, counts
 
 
 def decode(logit_source, *, B, W, V, n_total, dtype, top_k, cfg_scale=1.0, inv_temperature=1.0, reuse_tau=0.5,
            flags=FLAG_REUSE, seed=0, seq_base=0, max_steps=None, n_threads=1, trace=None, init_mode=INIT_RANDOM,
-           grid_width=0):
+           grid_width=0, refine=True):
     """Run the loop to the end.  `logit_source(window) -> (cond, uncond)` plays the model's forward pass.
     Returns (committed [B,n_total], steps, committed counts per step [steps,B])."""
     kcap = min(top_k, V)
@@ -186,7 +191,7 @@ def decode(logit_source, *, B, W, V, n_total, dtype, top_k, cfg_scale=1.0, inv_t
                      pos_base=w.pos_base, iteration=w.iteration, seed=seed, seq_base=seq_base, n_threads=n_threads)
         if trace is not None:
             trace.append((w, r))
-        w, counts = window_advance(w, r.accept_len, r.tokens, r.probs, V, n_total, seed, seq_base, init_mode, grid_width)
+        w, counts = window_advance(w, r.accept_len, r.tokens, r.probs, V, n_total, seed, seq_base, init_mode, grid_width, refine)
         history.append(counts)
         steps += 1
     return w.committed, steps, np.array(history, np.int32).reshape(steps, B)

@@ -155,3 +155,50 @@ def test_spatial_prior_needs_fewer_steps_than_random_on_a_repetitive_image(axis,
             total += s
         steps[m] = total
     assert steps[mode] < 0.8 * steps[loop.INIT_RANDOM], steps
+
+
+# ---- the "no refinement" ablation: unaccepted tokens are replaced by newly initialised ones ----
+
+def test_without_refinement_every_slot_behind_the_commit_is_new():
+    V, N, W = 200, 40, 7
+    src, source = _markov(V, N)
+    trace = []
+    loop.decode(source, B=2, W=W, V=V, n_total=N, dtype=oracle.F32, top_k=16, cfg_scale=3.0, seed=5, trace=trace, refine=False)
+    for w, _ in trace:
+        for b in range(2):
+            assert np.all(w.probs.cnt[b, :int(w.win_len[b])] == oracle.Q_UNIFORM)
+    trace = []
+    loop.decode(source, B=2, W=W, V=V, n_total=N, dtype=oracle.F32, top_k=16, cfg_scale=3.0, seed=5, trace=trace, refine=False,
+                init_mode=loop.INIT_REPEAT_LEFT, grid_width=5)
+    for n, (w, _) in enumerate(trace[1:]):
+        for b in range(2):
+            L, p0 = int(w.win_len[b]), int(w.pos_base[b])
+            assert np.all(w.drafts[b, :L] == w.committed[b, p0 - 1])      # the last committed token, repeated
+            assert np.all(w.probs.cnt[b, :L] == 1)
+
+
+def test_without_refinement_greedy_decoding_still_reaches_the_greedy_sequence():
+    V, N = 128, 30
+    out = []
+    for refine in (True, False):
+        src, source = _markov(V, N)
+        committed, steps, _ = loop.decode(source, B=1, W=8, V=V, n_total=N, dtype=oracle.F32, top_k=1, cfg_scale=3.0, seed=2,
+                                          refine=refine)
+        out.append(committed[0].tolist())
+    assert out[0] == out[1]
+
+
+def test_without_refinement_there_is_almost_no_acceleration():
+    # the paper's refinement ablation: replacing unaccepted tokens by new ones needs about one forward pass
+    # per token, refinement about half as many; a spatial prior helps a little when the image is flat
+    V, W, N = 512, 12, 96
+    src, source = _markov(V, N, states=16)
+    kw = dict(B=1, W=W, V=V, n_total=N, dtype=oracle.F32, top_k=64, cfg_scale=3.0, seed=3)
+    _, with_ref, _ = loop.decode(source, **kw)
+    _, without, _ = loop.decode(source, refine=False, **kw)
+    assert without >= 0.9 * N and without > 1.1 * with_ref, (with_ref, without)
+    flat = lambda seed: _pattern_source(V, W, 8, "left", seed=seed)
+    kw = dict(B=1, W=W, V=V, n_total=N, dtype=oracle.F32, top_k=64, seed=1)
+    _, rnd, _ = loop.decode(flat(1), refine=False, **kw)
+    _, rep, _ = loop.decode(flat(1), refine=False, init_mode=loop.INIT_REPEAT_LEFT, grid_width=8, **kw)
+    assert rnd >= 0.9 * N and rep < 0.5 * rnd, (rnd, rep)
