@@ -44,6 +44,8 @@ def parse_args():
                     help="--loop only: token initialisation (0 random, 1 repeat left, 2 repeat above, 3 sample left, 4 sample above)")
     ap.add_argument("--loop-source", default="markov", choices=["markov", "stripes"],
                     help="--loop only: synthetic logit source (first-order Markov chain, or an image of vertical stripes)")
+    ap.add_argument("--no-refine", action="store_true",
+                    help="--loop only: the no-refinement ablation (unaccepted slots are re-initialised, not carried over)")
     ap.add_argument("--graphs", action="store_true", help="--loop only: replay each iteration's kernels from a CUDA graph")
     ap.add_argument("--loop", action="store_true",
                     help="run the full decode loop of the 48x48 grid workload (cfg5) instead of the single-step benchmark")
@@ -453,7 +455,7 @@ def run_loop(args):
     noise_u = torch.randn(N, V, generator=g, device=dev).to(torch.bfloat16)
     G = 48
     dl = DecodeLoop(batch=1, window=W, vocab=V, n_total=N, logits_dtype=torch.bfloat16, top_k=K, cfg_scale=3.0, seed=5,
-                    init_mode=args.init_mode, grid_width=G, use_graphs=args.graphs, device=dev)
+                    init_mode=args.init_mode, grid_width=G, use_graphs=args.graphs, refine=not args.no_refine, device=dev)
     ar = torch.arange(W, device=dev)
     g.manual_seed(8)
     colours = torch.randperm(V, generator=g, device=dev)[:G]
@@ -499,7 +501,7 @@ def run_loop(args):
     lib_ms = sum(a.elapsed_time(b) for a, b in ev)
     print(json.dumps({"workload": "cfg5: decode loop, 2304 tokens, V=65536, W=32, bf16, CFG 3.0, top-K 2000, "
                                   + ("Markov source" if args.loop_source == "markov" else "vertical-stripes source"),
-                      "init_mode": args.init_mode, "grid_width": G, "cuda_graphs": bool(args.graphs), "steps": dl.steps, "tokens": N, "mean_committed_per_step": round(N / dl.steps, 4),
+                      "init_mode": args.init_mode, "grid_width": G, "cuda_graphs": bool(args.graphs), "refinement": not args.no_refine, "steps": dl.steps, "tokens": N, "mean_committed_per_step": round(N / dl.steps, 4),
                       "step_compression_S": round(N / dl.steps, 4), "library_ms_total": round(lib_ms, 3),
                       "library_us_per_step": round(1e3 * lib_ms / dl.steps, 2), "wall_s_including_logit_source": round(wall, 3),
                       "complete": bool((dl.committed >= 0).all().item())}), flush=True)

@@ -55,6 +55,10 @@ extern "C" {
 #define SJD_FLAG_DRAFT_ALL 2 /* no verification: draw every valid row from its own p (initial drafts; Section
                                 4.2 strategies that sample from a predicted distribution).  accept_len = 0. */
 
+#define SJD_FLAG_NO_REFINE 16 /* sjd_window_advance() only: the "no refinement" ablation of the paper's analysis
+                                section - nothing is carried over, every slot behind the committed tokens is
+                                newly initialised; sjd_step() ignores it                                   */
+
 #define SJD_FLAG_FORCE_GENERIC 4 /* diagnostics: use the any-shape multi-pass row kernel even where a
                                    single-pass kernel applies (results are identical)                    */
 #define SJD_FLAG_FORCE_TILES 8   /* diagnostics: skip the single-pass kernel that cuts a row into one id
@@ -211,15 +215,17 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
  *       SJD_INIT_REPEAT_ABOVE  the token at position p-G (p-1 when p < G), point-mass reference.  The token at an
  *                              earlier position is the committed one before the verified window, the step's
  *                              output token inside it, and a new slot's own initial token after it;
- *       SJD_INIT_SAMPLE_LEFT   a draw from the distribution of the last verified row (the nearest prediction to
- *                              the left), which also becomes the reference; fixed-point inverse CDF on Philox
+ *       SJD_INIT_SAMPLE_LEFT   a draw from the distribution the step predicted for position p-1, or from the last
+ *                              verified row's when p-1 lies behind the window (the nearest prediction to the
+ *                              left); it also becomes the reference; fixed-point inverse CDF on Philox
  *                              purpose 5, counter = (p, seq_base+b, iteration, 5), R = x0 | x1 << 32;
  *       SJD_INIT_SAMPLE_ABOVE  the same from the row of position p-G, stepping a further G back while that
- *                              position is itself a new slot; when it was verified before this step (its
+ *                              position lies behind the verified window; when it was verified before this step (its
  *                              distribution is gone) the committed token there with a point-mass reference;
  *                              when p < G (or the walk leaves the grid) as SJD_INIT_SAMPLE_LEFT.
  *     The paper names the strategies; the reference distributions, the fall-backs and the generator words are
- *     this library's;
+ *     this library's.  With SJD_FLAG_NO_REFINE no row is carried over: all win_len slots of the next window
+ *     are initialised as above, and only the committed tokens of this step count as known tokens;
  *   - updates win_len, pos_base, iteration in place: pos_base += c, win_len = min(W, n_total - pos_base),
  *     iteration += 1.  A sequence is finished when its win_len is 0.
  * params supplies B, W, V, top_k, seq_base, init_mode, grid_width and stream; its win_len/pos_base/iteration fields are not used

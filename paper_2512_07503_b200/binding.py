@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 SJD_F32, SJD_BF16 = 0, 1
-SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL, SJD_FLAG_FORCE_GENERIC, SJD_FLAG_FORCE_TILES = 1, 2, 4, 8
+SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL, SJD_FLAG_FORCE_GENERIC, SJD_FLAG_FORCE_TILES, SJD_FLAG_NO_REFINE = 1, 2, 4, 8, 16
 SJD_Q_UNIFORM = -1
 SJD_INIT_RANDOM, SJD_INIT_REPEAT_LEFT, SJD_INIT_REPEAT_ABOVE, SJD_INIT_SAMPLE_LEFT, SJD_INIT_SAMPLE_ABOVE = 0, 1, 2, 3, 4
 SJD_OUT_INVALID, SJD_OUT_ACCEPTED, SJD_OUT_RESIDUAL, SJD_OUT_REUSED, SJD_OUT_RESAMPLED = 0, 1, 2, 3, 4

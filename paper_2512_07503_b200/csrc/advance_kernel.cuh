@@ -20,6 +20,7 @@ struct AdvanceArgs {
   int B, W, V, kcap, n_total;
   int seq_base;
   int init_mode, grid_width;
+  int no_refine;  // 1: nothing is carried over, every slot behind the committed tokens is newly initialised
   uint32_t seed_lo, seed_hi;
   // result of the step that just ran
   const int32_t* accept_len;
@@ -82,7 +83,7 @@ __global__ void __launch_bounds__(NT) advance_rows_kernel(const AdvanceArgs a) {
     return;
   }
   const int src = i + c;
-  if (src < L) {
+  if (!a.no_refine && src < L) {
     // an unaccepted row moves up; its distribution of this iteration becomes the reference
     const size_t srow = (size_t)b * a.W + src;
     const int32_t* sid = a.step_ids + srow * a.kcap;
@@ -102,7 +103,8 @@ __global__ void __launch_bounds__(NT) advance_rows_kernel(const AdvanceArgs a) {
   // a new slot at absolute position p
   const int p = pos1 + i;
   const int G = a.grid_width;
-  const int end0 = pos0 + L;  // first position after the verified window
+  const int pred_end = pos0 + L;                      // first position the step made no prediction for
+  const int tok_end = a.no_refine ? pos1 : pred_end;  // first position whose token does not survive the step
   const int mode = a.init_mode;
   const bool above = (mode == kInitRepeatAbove || mode == kInitSampleAbove) && p >= G;
   const bool sample = mode == kInitSampleLeft || mode == kInitSampleAbove;
@@ -117,15 +119,18 @@ __global__ void __launch_bounds__(NT) advance_rows_kernel(const AdvanceArgs a) {
   // the position whose token (repeat) or prediction (sample) initialises this slot
   int r;
   if (!sample) {
-    // positions at or after end0 are new slots themselves: follow their own rule back into known tokens
+    // positions at or after tok_end are new slots themselves: follow their own rule back into known tokens
     r = above ? p - G : p - 1;
-    while (r >= end0) r -= (mode == kInitRepeatAbove && r >= G) ? G : 1;
-  } else if (above) {
-    r = p - G;
-    while (r >= end0) r -= G;
-    if (r < 0) r = end0 - 1;  // left the grid: the last verified row, as for "sample left"
+    while (r >= tok_end) r -= (mode == kInitRepeatAbove && r >= G) ? G : 1;
   } else {
-    r = end0 - 1;
+    const int left = min(p - 1, pred_end - 1);  // the prediction made for p-1, else the last one made
+    if (above) {
+      r = p - G;
+      while (r >= pred_end) r -= G;
+      if (r < 0) r = left;  // left the grid: as for "sample left"
+    } else {
+      r = left;
+    }
   }
   if (!sample || r < pos0) {
     if (threadIdx.x == 0) {

@@ -439,6 +439,7 @@ int fill_advance(sjd::AdvanceArgs* a, const sjd_params* P, int32_t n_total, uint
   a->seq_base = P->seq_base;
   a->init_mode = P->init_mode;
   a->grid_width = P->grid_width > 0 ? P->grid_width : 1;
+  a->no_refine = (P->flags & SJD_FLAG_NO_REFINE) ? 1 : 0;
   a->seed_lo = (uint32_t)(seed & 0xffffffffu);
   a->seed_hi = (uint32_t)(seed >> 32);
   a->win_len = win_len; a->pos_base = pos_base; a->iteration = iteration;

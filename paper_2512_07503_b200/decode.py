@@ -19,7 +19,7 @@ class DecodeLoop:
     def __init__(self, *, batch: int, window: int, vocab: int, n_total: int, logits_dtype: torch.dtype, top_k: int,
                  cfg_scale: float = 1.0, inv_temperature: float = 1.0, reuse_tau: float = 0.5, reuse: bool = True,
                  seed: int = 0, seq_base: int = 0, init_mode: int = B.SJD_INIT_RANDOM, grid_width: int = 1,
-                 use_graphs: bool = False, guidance: bool = True, device="cuda:0"):
+                 use_graphs: bool = False, guidance: bool = True, refine: bool = True, device="cuda:0"):
         self.B, self.W, self.V, self.N = batch, window, vocab, n_total
         self.kcap = min(top_k, vocab)
         self.seed, self.device = seed, torch.device(device)
@@ -39,7 +39,9 @@ class DecodeLoop:
         self.cur = 0
         proto = torch.empty(batch, window, vocab, dtype=logits_dtype, device=dev)
         self.params = B.make_params(proto, top_k=top_k, cfg_scale=cfg_scale, inv_temperature=inv_temperature,
-                                    reuse_tau=reuse_tau, flags=(B.SJD_FLAG_REUSE if reuse else 0), win_len=self.win_len,
+                                    reuse_tau=reuse_tau,
+                                    flags=(B.SJD_FLAG_REUSE if reuse else 0) | (0 if refine else B.SJD_FLAG_NO_REFINE),
+                                    win_len=self.win_len,
                                     pos_base=self.pos_base, iteration=self.iteration, status=self.status,
                                     seq_base=seq_base, init_mode=init_mode, grid_width=grid_width)
         del proto

@@ -14,7 +14,7 @@ DEV = "cuda:0"
 
 
 def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64, init_mode=0, grid_width=1, windows=False,
-          use_graphs=False):
+          use_graphs=False, refine=True):
     from paper_2512_07503_b200.decode import DecodeLoop
     src = wk.MarkovSource(V, N, dtype, states=states)
     flags = oracle.FLAG_REUSE if reuse else 0
@@ -22,11 +22,11 @@ def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64, init_mode=0,
     ref_committed, ref_steps, ref_counts = loop.decode(
         lambda w: src.logits(w.drafts, w.win_len, w.pos_base, w.committed), B=B, W=W, V=V, n_total=N, dtype=dtype,
         top_k=top_k, cfg_scale=3.0, flags=flags, seed=seed, n_threads=8, init_mode=init_mode, grid_width=grid_width,
-        trace=trace)
+        trace=trace, refine=refine)
 
     tdt = torch.bfloat16 if dtype == wk.BF16 else torch.float32
     dl = DecodeLoop(batch=B, window=W, vocab=V, n_total=N, logits_dtype=tdt, top_k=top_k, cfg_scale=3.0, reuse=reuse,
-                    seed=seed, init_mode=init_mode, grid_width=grid_width, use_graphs=use_graphs, device=DEV)
+                    seed=seed, init_mode=init_mode, grid_width=grid_width, use_graphs=use_graphs, refine=refine, device=DEV)
 
     def up(a):
         if dtype == wk.BF16:
@@ -80,6 +80,13 @@ def test_graph_replay_gives_the_same_trajectory(mode):
     got, ref = _both(2, 12, 8192, 70, 300, wk.BF16, init_mode=mode, grid_width=16, windows=True, use_graphs=True)
     assert got[1] == ref[1] and np.array_equal(got[2], ref[2]) and np.array_equal(got[0], ref[0])
     assert got[1] > 6
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2, 3, 4])
+def test_no_refinement_ablation_matches_the_oracle(mode):
+    # nothing is carried over: every slot behind the committed tokens is newly initialised
+    got, ref = _both(2, 10, 4096, 40, 64, wk.F32, init_mode=mode, grid_width=4, windows=True, refine=False)
+    assert got[1] == ref[1] and np.array_equal(got[2], ref[2]) and np.array_equal(got[0], ref[0])
 
 
 def test_random_initialisation_windows_match_the_oracle():
