@@ -18,7 +18,7 @@ _SRC = os.path.join(_HERE, "sjd_oracle.cpp")
 _HDR = os.path.join(_HERE, "sjd_oracle.h")
 _SO = os.path.join(_HERE, "libsjd_oracle.so")
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 FLAG_REUSE, FLAG_DRAFT_ALL = 1, 2
 PURPOSE_ACCEPT, PURPOSE_RESIDUAL, PURPOSE_REDRAFT, PURPOSE_INIT = 0, 1, 2, 3
 OUT_INVALID, OUT_ACCEPTED, OUT_RESIDUAL, OUT_REUSED, OUT_RESAMPLED = 0, 1, 2, 3, 4
@@ -66,6 +66,8 @@ def lib():
         L.orc_philox4x32_10.restype = None
         L.orc_uniform24.argtypes = [C.c_uint32]
         L.orc_uniform24.restype = C.c_float
+        L.orc_half_to_float.argtypes = [C.c_uint16]
+        L.orc_half_to_float.restype = C.c_float
         L.orc_row_probs.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_float,
                                     C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_row_probs.restype = C.c_int32
@@ -97,6 +99,10 @@ def philox4x32_10(ctr, key) -> np.ndarray:
     return out
 
 
+def half_to_float(bits: int) -> float:
+    return float(lib().orc_half_to_float(int(bits) & 0xFFFF))
+
+
 def uniform24(x: int) -> float:
     return float(lib().orc_uniform24(int(x) & 0xFFFFFFFF))
 
@@ -106,8 +112,8 @@ def _logits_view(a, dtype):
     if a is None:
         return None
     a = np.ascontiguousarray(a)
-    if dtype == BF16:
-        assert a.dtype == np.uint16, "bf16 logits are passed as their uint16 bit patterns"
+    if dtype in (BF16, F16):
+        assert a.dtype == np.uint16, "16-bit logits are passed as their uint16 bit patterns"
     else:
         assert a.dtype == np.float32
     return a

@@ -53,8 +53,20 @@ void draw(uint64_t seed, int32_t pos, int32_t b, int32_t iter, int32_t purpose, 
 
 float uniform24(uint32_t x) { return (float)(x >> 8) * (1.0f / 16777216.0f); }
 
+// IEEE 754 binary16: 1 sign bit, 5 exponent bits (bias 15), 10 fraction bits.  Every value is exactly
+// representable in fp32; written out case by case.
+float half_to_float(uint16_t h) {
+  const int sign = (h >> 15) & 1, e = (h >> 10) & 31, f = h & 1023;
+  double v;
+  if (e == 0) v = std::ldexp((double)f, -24);                  // zero and subnormals: f * 2^-10 * 2^-14
+  else if (e == 31) v = f == 0 ? (double)INFINITY : (double)NAN;
+  else v = std::ldexp(1.0 + (double)f / 1024.0, e - 15);
+  return (float)(sign ? -v : v);
+}
+
 // bf16 -> fp32 is exact: the 16 bits are the upper half of the fp32 pattern.
 float load_logit(const void* base, int32_t dtype, int64_t idx) {
+  if (dtype == ORC_F16) return half_to_float(((const uint16_t*)base)[idx]);
   if (dtype == ORC_BF16) {
     const uint32_t bits = (uint32_t)((const uint16_t*)base)[idx] << 16;
     float f;
@@ -327,6 +339,8 @@ extern "C" {
 
 void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) { philox(ctr, key, out); }
 
+float orc_half_to_float(uint16_t bits) { return half_to_float(bits); }
+
 float orc_uniform24(uint32_t x) { return uniform24(x); }
 
 int32_t orc_row_probs(const void* cond, const void* uncond, int32_t dtype, int32_t V, float cfg_scale,
@@ -357,7 +371,7 @@ int32_t orc_sjd_step(const void* logits_cond, const void* logits_uncond, const i
   if (!P || !logits_cond || !out_accept_len || !out_tokens || !out_probs) return -1;
   if (!out_probs->tok_prob || !out_probs->ids || !out_probs->vals || !out_probs->cnt) return -1;
   if (P->B < 0 || P->W < 1 || P->V < 1 || P->top_k < 1) return -2;
-  if (P->logits_dtype != ORC_F32 && P->logits_dtype != ORC_BF16) return -3;
+  if (P->logits_dtype != ORC_F32 && P->logits_dtype != ORC_BF16 && P->logits_dtype != ORC_F16) return -3;
   const bool draft_all = (P->flags & ORC_FLAG_DRAFT_ALL) != 0;
   if (!draft_all) {
     if (!drafts || !draft_probs) return -1;

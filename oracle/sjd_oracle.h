@@ -35,7 +35,7 @@
 extern "C" {
 #endif
 
-enum { ORC_F32 = 0, ORC_BF16 = 1 };
+enum { ORC_F32 = 0, ORC_BF16 = 1, ORC_F16 = 2 };
 
 /* flags */
 enum {
@@ -67,7 +67,7 @@ typedef struct {
 
 typedef struct {
   int32_t B, W, V;
-  int32_t logits_dtype;       /* ORC_F32 / ORC_BF16 (raw 16-bit patterns)                      */
+  int32_t logits_dtype;       /* ORC_F32 / ORC_BF16 / ORC_F16 (raw 16-bit patterns)            */
   int64_t stride_b, stride_w; /* element strides of both logits arrays; vocabulary contiguous  */
   float cfg_scale;            /* s of the guidance merge                                       */
   float inv_temperature;      /* 1/T, already rounded to float by the caller                   */
@@ -105,6 +105,9 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
 
 /* u = (x >> 8) * 2^-24, in [0,1). */
 float orc_uniform24(uint32_t x);
+
+/* Value of an IEEE 754 binary16 pattern, widened exactly to fp32 (the storage type of fp16 logits). */
+float orc_half_to_float(uint16_t bits);
 
 /* Sampling head for one row (Section 3.1; guidance weight and top-K of Section 5.1):
  * merged = uncond + s*(cond - uncond); y = merged / T; keep the kcap largest y (ties to the lower

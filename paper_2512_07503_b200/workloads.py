@@ -18,7 +18,7 @@ from dataclasses import dataclass, replace
 
 import numpy as np
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 
 
 @dataclass(frozen=True)
@@ -104,10 +104,14 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 
 
 def _store(x: np.ndarray, dtype: int) -> np.ndarray:
+    if dtype == F16:   # IEEE half precision, round to nearest even; kept as uint16 patterns like bf16
+        return np.ascontiguousarray(x, dtype=np.float32).astype(np.float16).view(np.uint16)
     return to_bf16_bits(x) if dtype == BF16 else np.ascontiguousarray(x, dtype=np.float32)
 
 
 def _as_f32(x: np.ndarray, dtype: int) -> np.ndarray:
+    if dtype == F16:
+        return x.view(np.float16).astype(np.float32)
     return bf16_bits_to_f32(x) if dtype == BF16 else x
 
 

@@ -146,3 +146,22 @@ def test_sum_and_count(V, K):
     ids, vals, _ = oracle.row_probs(c, u, oracle.F32, 3.0, np.float32(1 / 0.9), K)
     assert len(ids) == min(K, V)
     assert abs(float(vals.astype(np.float64).sum()) - 1.0) < 1e-6
+
+
+def test_half_precision_patterns_decode_like_numpy_for_all_65536_values():
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    ref = bits.view(np.float16).astype(np.float32)
+    got = np.array([oracle.half_to_float(int(b)) for b in bits], dtype=np.float32)
+    nan = np.isnan(ref)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan].view(np.uint32), ref[~nan].view(np.uint32))   # bit for bit, signed zeros included
+
+
+def test_fp16_rows_equal_the_same_values_given_as_fp32():
+    rng = np.random.default_rng(5)
+    V = 1024
+    c16 = (rng.standard_normal(V) * 3).astype(np.float16)
+    u16 = (c16.astype(np.float32) + rng.standard_normal(V).astype(np.float32)).astype(np.float16)
+    a = oracle.row_probs(c16.view(np.uint16), u16.view(np.uint16), oracle.F16, 3.0, 1.0, 50)
+    b = oracle.row_probs(c16.astype(np.float32), u16.astype(np.float32), oracle.F32, 3.0, 1.0, 50)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
