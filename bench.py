@@ -53,7 +53,7 @@ def parse_args():
 
 
 def workload_config(wl, n_gpus):
-    return {"workload": f"{wl.name}: B={wl.B} W={wl.W} V={wl.V} {'bf16' if wl.dtype == 1 else 'fp32'} logits, "
+    return {"workload": f"{wl.name}: B={wl.B} W={wl.W} V={wl.V} {('fp32', 'bf16', 'fp16')[wl.dtype]} logits, "
                         f"CFG {wl.cfg_scale}, T {wl.temperature}, top-K {wl.top_k}, reuse tau {wl.reuse_tau}",
             "B_per_gpu": wl.B, "W": wl.W, "V": wl.V, "top_k": wl.top_k, "global_batch": wl.B * n_gpus,
             "parallelism": f"replicas over B x{n_gpus}, no collective",
@@ -63,7 +63,7 @@ def workload_config(wl, n_gpus):
 def algorithmic_bytes(wl) -> int:
     """Bytes the method itself must move per step: both logits tensors read, the sparse distributions and
     per-position results written, one previous-iteration sparse row per sequence read."""
-    esize = 2 if wl.dtype == 1 else 4
+    esize = 4 if wl.dtype == 0 else 2
     rows = wl.B * wl.W
     return rows * (2 * wl.V * esize + 8 * wl.kcap + 16) + wl.B * 8 * wl.kcap
 
@@ -134,7 +134,7 @@ def device_inputs(wl, device, seed):
     import torch
     g = torch.Generator(device=device)
     g.manual_seed(seed)
-    dt = torch.bfloat16 if wl.dtype == 1 else torch.float32
+    dt = {0: torch.float32, 1: torch.bfloat16, 2: torch.float16}[wl.dtype]
     shape = (wl.B, wl.W, wl.V)
     cond = torch.randn(shape, generator=g, device=device, dtype=torch.float32) * wl.sigma
     if wl.peaks > 0:
@@ -355,7 +355,7 @@ def host_arrays(dset):
     wl = dset.wl
 
     def logits(t):
-        if wl.dtype == 1:
+        if wl.dtype != 0:
             return t.view(torch.int16).cpu().numpy().view(np.uint16)
         return t.cpu().numpy()
 

@@ -49,6 +49,7 @@ extern "C" {
 /* logits_dtype */
 #define SJD_F32 0
 #define SJD_BF16 1
+#define SJD_F16 2 /* IEEE half precision */
 
 /* flags */
 #define SJD_FLAG_REUSE 1     /* Eq. reuse (SJD++); clear = Eq. refine-sjd (SJD)                              */
@@ -114,7 +115,7 @@ typedef struct {
 typedef struct {
   int32_t struct_size;        /* sizeof(sjd_params)                                                        */
   int32_t B, W, V;            /* sequences, window rows, vocabulary                                        */
-  int32_t logits_dtype;       /* SJD_F32 or SJD_BF16                                                       */
+  int32_t logits_dtype;       /* SJD_F32, SJD_BF16 or SJD_F16                                              */
   int64_t stride_b, stride_w; /* element strides of BOTH logits tensors; the vocabulary axis is contiguous;
                                  stride * element size must be a multiple of 16 bytes                      */
   float cfg_scale;            /* s; unused when logits_uncond is NULL                                      */

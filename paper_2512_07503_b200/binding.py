@@ -14,7 +14,7 @@ import torch
 
 from . import build as _build
 
-SJD_F32, SJD_BF16 = 0, 1
+SJD_F32, SJD_BF16, SJD_F16 = 0, 1, 2
 SJD_FLAG_REUSE, SJD_FLAG_DRAFT_ALL, SJD_FLAG_FORCE_GENERIC, SJD_FLAG_FORCE_TILES, SJD_FLAG_NO_REFINE = 1, 2, 4, 8, 16
 SJD_Q_UNIFORM = -1
 SJD_INIT_RANDOM, SJD_INIT_REPEAT_LEFT, SJD_INIT_REPEAT_ABOVE, SJD_INIT_SAMPLE_LEFT, SJD_INIT_SAMPLE_ABOVE = 0, 1, 2, 3, 4
@@ -151,15 +151,17 @@ def make_params(logits: torch.Tensor, *, top_k: int, cfg_scale: float = 1.0, inv
                 status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
                 stream: Optional[torch.cuda.Stream] = None, seq_base: int = 0, init_mode: int = 0,
                 grid_width: int = 1) -> sjd_params:
-    """Fill an ``sjd_params`` from a [B,W,V] logits tensor (fp32 or bf16, vocabulary axis contiguous)."""
+    """Fill an ``sjd_params`` from a [B,W,V] logits tensor (fp32, bf16 or fp16, vocabulary axis contiguous)."""
     if logits.dim() != 3 or logits.stride(2) != 1:
         raise SjdError("logits must be [B,W,V] with a contiguous vocabulary axis")
     if logits.dtype == torch.float32:
         dt = SJD_F32
     elif logits.dtype == torch.bfloat16:
         dt = SJD_BF16
+    elif logits.dtype == torch.float16:
+        dt = SJD_F16
     else:
-        raise SjdError("logits must be float32 or bfloat16")
+        raise SjdError("logits must be float32, bfloat16 or float16")
     B, W, V = logits.shape
     p = sjd_params()
     p.struct_size = C.sizeof(sjd_params)

@@ -3,6 +3,7 @@
 // any group of NT threads synchronised by a named barrier.
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -74,6 +75,8 @@ __device__ __forceinline__ float merge_logit(float c, float u, float s, float in
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+// the two IEEE half-precision values of a 32-bit word, widened exactly
+__device__ __forceinline__ float2 f16_pair(uint32_t w) { return __half22float2(*reinterpret_cast<const __half2*>(&w)); }
 
 // Eight consecutive logits starting at element `e` (a multiple of 8) of a row, converted to fp32.
 template <int DTYPE>
@@ -82,6 +85,10 @@ __device__ __forceinline__ void load8(const void* __restrict__ row, int e, float
     const uint4 w = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(row) + e));
     x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
     x[4] = bf16_lo(w.z); x[5] = bf16_hi(w.z); x[6] = bf16_lo(w.w); x[7] = bf16_hi(w.w);
+  } else if (DTYPE == 2) {
+    const uint4 w = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(row) + e));
+    const float2 a = f16_pair(w.x), b = f16_pair(w.y), c = f16_pair(w.z), d = f16_pair(w.w);
+    x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y; x[4] = c.x; x[5] = c.y; x[6] = d.x; x[7] = d.y;
   } else {
     const float4 a = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(row) + e));
     const float4 b = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(row) + e) + 1);

@@ -47,7 +47,7 @@ struct GenericSmem {
 
 __device__ __forceinline__ const void* row_ptr(const void* base, int dtype, int64_t elem) {
   return base == nullptr ? nullptr
-                         : static_cast<const void*>(static_cast<const char*>(base) + elem * (dtype == 1 ? 2 : 4));
+                         : static_cast<const void*>(static_cast<const char*>(base) + elem * (dtype == 0 ? 4 : 2));
 }
 
 // One row through global memory.  All NT threads of the group call it with the same arguments.

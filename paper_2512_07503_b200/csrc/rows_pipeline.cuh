@@ -165,17 +165,17 @@ struct RowSchedule {
 
 template <int DTYPE>
 struct PipeTraits {
-  static constexpr int kElemBytes = DTYPE == 1 ? 2 : 4;
+  static constexpr int kElemBytes = DTYPE == 0 ? 4 : 2;
   static constexpr int kTileBytes = kTileElems * kElemBytes;
   static constexpr int kTilesPerStage = kStageArrayBytes / kTileBytes;  // 16 (bf16) or 8 (fp32)
   static constexpr int kStageBytes = 2 * kStageArrayBytes;
 };
 
-// Element index inside a tile of the j-th value a lane holds.  bf16: 8 consecutive elements per lane
+// Element index inside a tile of the j-th value a lane holds.  bf16 / fp16: 8 consecutive elements per lane
 // (one 16-byte load).  fp32: elements 4*lane..+3 and 128+4*lane..+3 (two conflict-free 16-byte loads).
 template <int DTYPE>
 __device__ __forceinline__ int tile_elem(int lane, int j) {
-  if (DTYPE == 1) return lane * 8 + j;
+  if (DTYPE != 0) return lane * 8 + j;
   return j < 4 ? lane * 4 + j : 128 + lane * 4 + (j - 4);
 }
 
@@ -188,17 +188,17 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 // A thread's share of a staged tile as it lies in shared memory: 8 logits of each array.
 template <int DTYPE>
 struct RawTile {
-  uint4 c[DTYPE == 1 ? 1 : 2];
-  uint4 u[DTYPE == 1 ? 1 : 2];
+  uint4 c[DTYPE != 0 ? 1 : 2];
+  uint4 u[DTYPE != 0 ? 1 : 2];
 };
 
 template <int DTYPE, bool has_u>
 __device__ __forceinline__ void load_raw(uint32_t ctile, uint32_t utile, int lane, RawTile<DTYPE>& r) {
   r.c[0] = lds128(ctile + lane * 16);
-  if (DTYPE != 1) r.c[DTYPE == 1 ? 0 : 1] = lds128(ctile + 512 + lane * 16);
+  if (DTYPE == 0) r.c[DTYPE != 0 ? 0 : 1] = lds128(ctile + 512 + lane * 16);
   if (has_u) {
     r.u[0] = lds128(utile + lane * 16);
-    if (DTYPE != 1) r.u[DTYPE == 1 ? 0 : 1] = lds128(utile + 512 + lane * 16);
+    if (DTYPE == 0) r.u[DTYPE != 0 ? 0 : 1] = lds128(utile + 512 + lane * 16);
   }
 }
 
@@ -217,12 +217,21 @@ __device__ __forceinline__ void merge_raw(const RawTile<DTYPE>& r, uint64_t s2, 
       u[0] = pack2(bf16_lo(v.x), bf16_hi(v.x)); u[1] = pack2(bf16_lo(v.y), bf16_hi(v.y));
       u[2] = pack2(bf16_lo(v.z), bf16_hi(v.z)); u[3] = pack2(bf16_lo(v.w), bf16_hi(v.w));
     }
+  } else if (DTYPE == 2) {
+    const uint4 w = r.c[0];
+    const float2 c0 = f16_pair(w.x), c1 = f16_pair(w.y), c2 = f16_pair(w.z), c3 = f16_pair(w.w);
+    c[0] = pack2(c0.x, c0.y); c[1] = pack2(c1.x, c1.y); c[2] = pack2(c2.x, c2.y); c[3] = pack2(c3.x, c3.y);
+    if (has_u) {
+      const uint4 v = r.u[0];
+      const float2 u0 = f16_pair(v.x), u1 = f16_pair(v.y), u2 = f16_pair(v.z), u3 = f16_pair(v.w);
+      u[0] = pack2(u0.x, u0.y); u[1] = pack2(u1.x, u1.y); u[2] = pack2(u2.x, u2.y); u[3] = pack2(u3.x, u3.y);
+    }
   } else {
-    const uint4 a = r.c[0], b = r.c[DTYPE == 1 ? 0 : 1];
+    const uint4 a = r.c[0], b = r.c[DTYPE != 0 ? 0 : 1];
     c[0] = (uint64_t)a.x | ((uint64_t)a.y << 32); c[1] = (uint64_t)a.z | ((uint64_t)a.w << 32);
     c[2] = (uint64_t)b.x | ((uint64_t)b.y << 32); c[3] = (uint64_t)b.z | ((uint64_t)b.w << 32);
     if (has_u) {
-      const uint4 p = r.u[0], q = r.u[DTYPE == 1 ? 0 : 1];
+      const uint4 p = r.u[0], q = r.u[DTYPE != 0 ? 0 : 1];
       u[0] = (uint64_t)p.x | ((uint64_t)p.y << 32); u[1] = (uint64_t)p.z | ((uint64_t)p.w << 32);
       u[2] = (uint64_t)q.x | ((uint64_t)q.y << 32); u[3] = (uint64_t)q.z | ((uint64_t)q.w << 32);
     }

@@ -133,7 +133,7 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
   constexpr int NT_F = kRangeThreads;
   constexpr int BAR_F = 1;
   constexpr uint32_t kStride = NT_F * 8;         // bytes between consecutive entries of one filter thread
-  constexpr int TI = DTYPE == 1 ? 4 : 2;          // groups of eight elements per stage and thread
+  constexpr int TI = DTYPE != 0 ? 4 : 2;          // groups of eight elements per stage and thread
   constexpr int NS = kRangeRingStages;
   const int lane = tid & 31;
   const int mask_words = cfg.mask_words;
@@ -154,15 +154,15 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
 
   // the j-th group of eight elements of this thread in the staged slice at `stage`
   auto load_group = [&](uint32_t stage, int j, RawTile<DTYPE>& r) {
-    if (DTYPE == 1) {
+    if (DTYPE != 0) {
       r.c[0] = lds128(stage + my_row + (((uint32_t)j ^ swz) << 4));
       if (HAS_U) r.u[0] = lds128(stage + kRangeStageBytes + my_row + (((uint32_t)j ^ swz) << 4));
     } else {
       r.c[0] = lds128(stage + my_row + (((uint32_t)(2 * j) ^ swz) << 4));
-      r.c[DTYPE == 1 ? 0 : 1] = lds128(stage + my_row + (((uint32_t)(2 * j + 1) ^ swz) << 4));
+      r.c[DTYPE != 0 ? 0 : 1] = lds128(stage + my_row + (((uint32_t)(2 * j + 1) ^ swz) << 4));
       if (HAS_U) {
         r.u[0] = lds128(stage + kRangeStageBytes + my_row + (((uint32_t)(2 * j) ^ swz) << 4));
-        r.u[DTYPE == 1 ? 0 : 1] = lds128(stage + kRangeStageBytes + my_row + (((uint32_t)(2 * j + 1) ^ swz) << 4));
+        r.u[DTYPE != 0 ? 0 : 1] = lds128(stage + kRangeStageBytes + my_row + (((uint32_t)(2 * j + 1) ^ swz) << 4));
       }
     }
   };
@@ -390,7 +390,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   constexpr int BAR_P = 2;  // named barrier of the finisher warps (the filter warps use 1)
   constexpr int kFinItems = kKcapMax / NT_P;
   constexpr int NS = kRangeRingStages;
-  constexpr int BW = 64 / (DTYPE == 1 ? 2 : 4);  // elements per stage and range
+  constexpr int BW = 64 / (DTYPE != 0 ? 2 : 4);  // elements per stage and range
   static_assert(NT_F == NF * 32 && kFinItems == 8, "group sizes");
   extern __shared__ unsigned char smem_raw[];
   RangeSmem sm = carve_range_smem(smem_raw, cfg.mask_words);

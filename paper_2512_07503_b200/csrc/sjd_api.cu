@@ -70,7 +70,7 @@ int sample_rank(double a) {
 bool plan_pipeline(const sjd_params* P, int kcap, sjd::PipeCfg* cfg, size_t* smem) {
   const int V = P->V;
   if (kcap > sjd::kKcapMax || V % sjd::kTileElems != 0) return false;
-  const int tile_bytes = sjd::kTileElems * (P->logits_dtype == SJD_BF16 ? 2 : 4);
+  const int tile_bytes = sjd::kTileElems * (P->logits_dtype == SJD_F32 ? 4 : 2);
   const int tps = sjd::kStageArrayBytes / tile_bytes;
   const int tiles = V / sjd::kTileElems;
   const int vwords = V / 32;
@@ -130,7 +130,7 @@ EncodeTiledFn encode_tiled_fn() {
 // Same sampling rule as plan_pipeline; the sample is stage 0, i.e. 1/S of the row.
 bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem, bool need_encoder = true) {
   const int V = P->V;
-  const int es = P->logits_dtype == SJD_BF16 ? 2 : 4;
+  const int es = P->logits_dtype == SJD_F32 ? 4 : 2;
   const int bw = 64 / es;  // elements per stage and range
   if (kcap > sjd::kKcapMax || V % sjd::kRangeThreads != 0) return false;
   const int R = V / sjd::kRangeThreads;
@@ -165,12 +165,14 @@ bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem
 
 // Tensor map over one logits array: dims {R ids, 256 ranges, rows}, box {64 bytes, 256, 1}, 64-byte swizzle.
 bool make_range_map(CUtensorMap* map, const void* base, const sjd_params* P, const sjd::RangeCfg& cfg) {
-  const int es = P->logits_dtype == SJD_BF16 ? 2 : 4;
+  const int es = P->logits_dtype == SJD_F32 ? 4 : 2;
   const cuuint64_t dims[3] = {(cuuint64_t)cfg.range_len, (cuuint64_t)sjd::kRangeThreads, (cuuint64_t)P->B * (cuuint64_t)P->W};
   const cuuint64_t strides[2] = {(cuuint64_t)cfg.range_len * es, (cuuint64_t)P->stride_w * es};
   const cuuint32_t box[3] = {(cuuint32_t)(64 / es), (cuuint32_t)sjd::kRangeThreads, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = encode_tiled_fn()(map, P->logits_dtype == SJD_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+  const CUresult r = encode_tiled_fn()(map, P->logits_dtype == SJD_BF16  ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                       : P->logits_dtype == SJD_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                                    : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
                                        3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                        CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -299,8 +301,8 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
   const bool draft_all = (P->flags & SJD_FLAG_DRAFT_ALL) != 0;
   if (!draft_all && (!drafts || check_probs(draft_probs) != SJD_OK)) return SJD_ERR_NULL;
   if (P->B < 0 || P->W < 1 || P->W > SJD_W_MAX || P->V < 8 || (P->V % 8) != 0 || P->top_k < 1) return SJD_ERR_SHAPE;
-  if (P->logits_dtype != SJD_F32 && P->logits_dtype != SJD_BF16) return SJD_ERR_DTYPE;
-  const int64_t esize = P->logits_dtype == SJD_BF16 ? 2 : 4;
+  if (P->logits_dtype != SJD_F32 && P->logits_dtype != SJD_BF16 && P->logits_dtype != SJD_F16) return SJD_ERR_DTYPE;
+  const int64_t esize = P->logits_dtype == SJD_F32 ? 4 : 2;
   if (!aligned16(logits_cond) || (logits_uncond && !aligned16(logits_uncond)) || (P->stride_b * esize) % 16 != 0 ||
       (P->stride_w * esize) % 16 != 0 || P->stride_w < P->V || P->stride_b < 0)
     return SJD_ERR_ALIGN;
@@ -349,16 +351,20 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
     if (fast && plan_ranges(P, kcap, &rcfg, &smem) && make_range_map(&map_c, logits_cond, P, rcfg) &&
         make_range_map(&map_u, logits_uncond ? logits_uncond : logits_cond, P, rcfg)) {
       const int grid = rows < sm_count() ? rows : sm_count();
-      e = P->logits_dtype == SJD_BF16 ? launch_ranges<1>(ra, rcfg, map_c, map_u, smem, grid, stream)
-                                      : launch_ranges<0>(ra, rcfg, map_c, map_u, smem, grid, stream);
+      e = P->logits_dtype == SJD_BF16  ? launch_ranges<1>(ra, rcfg, map_c, map_u, smem, grid, stream)
+          : P->logits_dtype == SJD_F16 ? launch_ranges<2>(ra, rcfg, map_c, map_u, smem, grid, stream)
+                                       : launch_ranges<0>(ra, rcfg, map_c, map_u, smem, grid, stream);
     } else if (!(P->flags & SJD_FLAG_FORCE_GENERIC) && plan_pipeline(P, kcap, &cfg, &smem)) {
       const int grid = rows < sm_count() ? rows : sm_count();
-      e = P->logits_dtype == SJD_BF16 ? launch_pipeline<1>(ra, cfg, smem, grid, stream)
-                                      : launch_pipeline<0>(ra, cfg, smem, grid, stream);
+      e = P->logits_dtype == SJD_BF16  ? launch_pipeline<1>(ra, cfg, smem, grid, stream)
+          : P->logits_dtype == SJD_F16 ? launch_pipeline<2>(ra, cfg, smem, grid, stream)
+                                       : launch_pipeline<0>(ra, cfg, smem, grid, stream);
     } else {
       const int grid = rows < 4 * sm_count() ? rows : 4 * sm_count();
       e = P->logits_dtype == SJD_BF16
               ? launch_after(sjd::rows_generic_kernel<1, kGenericThreads>, dim3((unsigned)grid), dim3(kGenericThreads), 0, stream, true, ra)
+          : P->logits_dtype == SJD_F16
+              ? launch_after(sjd::rows_generic_kernel<2, kGenericThreads>, dim3((unsigned)grid), dim3(kGenericThreads), 0, stream, true, ra)
               : launch_after(sjd::rows_generic_kernel<0, kGenericThreads>, dim3((unsigned)grid), dim3(kGenericThreads), 0, stream, true, ra);
     }
     if (e != cudaSuccess) return cuda_fail(e, "row kernel launch");
@@ -456,8 +462,8 @@ int sjd_row_kernel(const sjd_params* P) {
   if (!P) return SJD_ERR_NULL;
   if (P->struct_size != (int32_t)sizeof(sjd_params)) return SJD_ERR_STRUCT;
   if (P->B < 0 || P->W < 1 || P->W > SJD_W_MAX || P->V < 8 || (P->V % 8) != 0 || P->top_k < 1) return SJD_ERR_SHAPE;
-  if (P->logits_dtype != SJD_F32 && P->logits_dtype != SJD_BF16) return SJD_ERR_DTYPE;
-  const int64_t esize = P->logits_dtype == SJD_BF16 ? 2 : 4;
+  if (P->logits_dtype != SJD_F32 && P->logits_dtype != SJD_BF16 && P->logits_dtype != SJD_F16) return SJD_ERR_DTYPE;
+  const int64_t esize = P->logits_dtype == SJD_F32 ? 4 : 2;
   if ((P->stride_b * esize) % 16 != 0 || (P->stride_w * esize) % 16 != 0 || P->stride_w < P->V || P->stride_b < 0)
     return SJD_ERR_ALIGN;
   const int kcap = P->top_k < P->V ? P->top_k : P->V;

@@ -49,13 +49,13 @@ int sjd_host_ctx_create(const sjd_params* s, sjd_host_ctx** out_ctx) {
   if (!s || !out_ctx) return SJD_ERR_NULL;
   *out_ctx = nullptr;
   if (s->B < 1 || s->W < 1 || s->W > SJD_W_MAX || s->V < 8 || (s->V % 8) != 0 || s->top_k < 1) return SJD_ERR_SHAPE;
-  if (s->logits_dtype != SJD_F32 && s->logits_dtype != SJD_BF16) return SJD_ERR_DTYPE;
+  if (s->logits_dtype != SJD_F32 && s->logits_dtype != SJD_BF16 && s->logits_dtype != SJD_F16) return SJD_ERR_DTYPE;
   sjd_host_ctx* c = static_cast<sjd_host_ctx*>(std::calloc(1, sizeof(sjd_host_ctx)));
   if (!c) return SJD_ERR_CUDA;
   c->B = s->B; c->W = s->W; c->V = s->V; c->dtype = s->logits_dtype; c->top_k = s->top_k;
   c->kcap = s->top_k < s->V ? s->top_k : s->V;
   c->rows = (size_t)s->B * s->W;
-  c->logits_bytes = c->rows * (size_t)s->V * (s->logits_dtype == SJD_BF16 ? 2 : 4);
+  c->logits_bytes = c->rows * (size_t)s->V * (s->logits_dtype == SJD_F32 ? 4 : 2);
   sjd_params shape;
   std::memset(&shape, 0, sizeof(shape));
   shape.B = s->B; shape.W = s->W;

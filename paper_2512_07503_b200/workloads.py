@@ -27,7 +27,7 @@ class Workload:
     B: int
     W: int
     V: int
-    dtype: int            # F32 or BF16
+    dtype: int            # F32, BF16 or F16
     sigma: float          # std of the conditional logits
     peaks: int            # tokens per row boosted by `boost`
     boost: float
@@ -81,6 +81,7 @@ def _sweep():
     out["v32k"] = base.scaled(name="v32k", V=32768, seed=301)
     out["v16k"] = base.scaled(name="v16k", V=16384, seed=302)
     out["v16k_f32"] = base.scaled(name="v16k_f32", V=16384, dtype=F32, seed=303)
+    out["f16"] = base.scaled(name="f16", dtype=F16, seed=304)
     return out
 
 

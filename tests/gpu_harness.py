@@ -18,6 +18,8 @@ def to_device_logits(a: np.ndarray, dtype: int) -> torch.Tensor:
         return None
     if dtype == wk.BF16:
         return torch.from_numpy(a.view(np.int16)).to(DEV).view(torch.bfloat16)
+    if dtype == wk.F16:
+        return torch.from_numpy(a.view(np.int16)).to(DEV).view(torch.float16)
     return torch.from_numpy(a).to(DEV)
 
 

@@ -250,3 +250,24 @@ def test_every_row_kernel_gives_the_same_answer(force):
     _run(wk.CONFIGS["cfg2"].scaled(W=6), flags=oracle.FLAG_REUSE | force)
     _run(wk.CONFIGS["cfg2"].scaled(W=6, top_k=1000), flags=oracle.FLAG_REUSE | force)   # a shape the tile kernel takes
     _run(wk.CONFIGS["cfg3"].scaled(B=6), flags=oracle.FLAG_REUSE | force)
+
+
+@pytest.mark.parametrize("V,K", [(16384, 300), (4096, 64), (1032, 7)])
+def test_fp16_all_classes_of_bit_patterns(V, K):
+    # logits taken from random 16-bit patterns: normal, subnormal, zero of both signs, infinities, NaNs
+    from gpu_harness import check_parity, oracle_prime, step_kwargs
+    wl = wk.CONFIGS["cfg2"].scaled(B=2, W=4, V=V, top_k=K, dtype=wk.F16, seed=77)
+    inp = wk.make_step_inputs(wl)
+    rng = np.random.default_rng(V)
+    for arr in (inp.cond, inp.prev_cond):
+        raw = rng.integers(0, 65536, size=arr.shape, dtype=np.uint32).astype(np.uint16)
+        pick = rng.random(arr.shape) < 0.3
+        arr[pick] = raw[pick]
+        if V == 1032:
+            arr[..., 5] = 0x7C00      # one +inf per row in the smallest case
+    prev = oracle_prime(inp)
+    check_parity(inp.cond, None, prev.tokens, prev.probs, step_kwargs(inp), inp.win_len)
+    wl2 = wk.CONFIGS["cfg2"].scaled(B=2, W=4, V=V, top_k=K, dtype=wk.F16, seed=78)
+    inp2 = wk.make_step_inputs(wl2)
+    prev2 = oracle_prime(inp2)
+    check_parity(inp2.cond, inp2.uncond, prev2.tokens, prev2.probs, step_kwargs(inp2), inp2.win_len)

@@ -19,7 +19,7 @@ def _case(seed):
         V = int(rng.choice([2048, 4096, 6144, 10240, 18432])) if rng.random() < 0.5 else 8 * int(rng.integers(1, 1500))
     else:
         V = 256 * int(rng.integers(8, 200))
-    dtype = wk.BF16 if rng.random() < 0.6 else wk.F32
+    dtype = [wk.BF16, wk.F32, wk.F16][int(rng.choice(3, p=[0.45, 0.3, 0.25]))]
     K = int(min(V, rng.choice([1, 2, 7, 50, 64, 300, 777, 1000, 2000, 2048, 2500])))
     W = int(rng.integers(1, 20))
     B = int(rng.integers(1, 4))
@@ -38,4 +38,4 @@ def test_random_case_matches_the_oracle(seed):
     inp = wk.make_step_inputs(wl)
     prev = oracle_prime(inp)
     rep, got, ref = check_parity(inp.cond, inp.uncond, prev.tokens, prev.probs, step_kwargs(inp), inp.win_len)
-    print(wl.name, wl.V, wl.top_k, wl.W, wl.B, "bf16" if wl.dtype == wk.BF16 else "f32", rep.summary())
+    print(wl.name, wl.V, wl.top_k, wl.W, wl.B, ("f32", "bf16", "f16")[wl.dtype], rep.summary())
