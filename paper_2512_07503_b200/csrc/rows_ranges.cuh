@@ -215,8 +215,7 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
     const float scale = (refine && range > 0.0f) ? __fdiv_rn((float)kHistBins - 0.5f, range) : 0.0f;
 
     uint32_t cur = list_base;  // shared-memory address of the thread's next free entry
-    uint32_t imw = 0;          // inverted hit bits of the last (it & 7) groups
-    int it = 0;                // groups of eight this thread has filtered in this row
+    uint32_t imw = 0;          // inverted hit bits of the groups filtered since the last full mask word
     bool overflow = false;
     // One group: four pairs.  A pair is always stored at the cursor; the cursor moves on only for a hit,
     // i.e. when max(pair) >= thr.  A pair of NaNs and -inf never hit.
@@ -239,9 +238,12 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
             : "f"(m), "f"(thr), "r"(kStride), "r"(8u >> k));
       }
       cur = d;
-      ++it;
-      if ((it & 7) == 0) {
-        if ((it >> 3) <= mask_words) sm.masks[(size_t)((it >> 3) - 1) * NT_F + tid] = imw;
+    };
+    // after stage s the thread has filtered (s + 1) TI groups; every eight groups fill one mask word
+    auto end_stage = [&](int s) {
+      const int done = (s + 1) * TI;
+      if ((done & 7) == 0) {
+        if ((done >> 3) <= mask_words) sm.masks[(size_t)((done >> 3) - 1) * NT_F + tid] = imw;
         imw = 0;
       }
     };
@@ -253,6 +255,7 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
       load_group(stage0, j, raw);
       filter_group(raw, sample_thr);
     }
+    end_stage(0);
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.empty[slot]);
     if (++slot == NS) {
@@ -299,6 +302,7 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
         for (int j = 0; j < TI; ++j) load_group(stage, j, raw[j]);
 #pragma unroll
         for (int j = 0; j < TI; ++j) filter_group(raw[j], tau0);
+        end_stage(s);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.empty[slot]);
@@ -311,6 +315,7 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
     // Threads own ascending id ranges and meet their ids in ascending order, so writing the runs one
     // after the other yields the candidates in ascending id order.
     {
+      const int it = cfg.stages * TI;  // groups of eight this thread has filtered in this row
       const int rem = it & 7;
       int w = it >> 3;
       if (rem != 0 && w < mask_words) {
