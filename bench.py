@@ -305,7 +305,7 @@ def run_ours(args):
 
 # DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture, per workload;
 # the capture is summarised under profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES = {"cfg4": 281_000_000}
+NCU_TRAFFIC_BYTES = {"cfg4": 280_100_000}
 
 
 def run_e2e(sjd, wl, dset, device, n, world, tokens_per_step, barrier):
