@@ -137,6 +137,8 @@ def device_inputs(wl, device, seed):
     dt = {0: torch.float32, 1: torch.bfloat16, 2: torch.float16}[wl.dtype]
     shape = (wl.B, wl.W, wl.V)
     cond = torch.randn(shape, generator=g, device=device, dtype=torch.float32) * wl.sigma
+    if wl.row_spread > 0:
+        cond *= torch.exp(wl.row_spread * (2 * torch.rand(wl.B, wl.W, 1, generator=g, device=device) - 1))
     if wl.peaks > 0:
         idx = torch.rand(wl.B, wl.W, wl.V, generator=g, device=device).topk(wl.peaks, dim=-1).indices
         cond.scatter_add_(2, idx, torch.full(idx.shape, wl.boost, device=device))

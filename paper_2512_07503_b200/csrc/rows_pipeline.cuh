@@ -474,8 +474,7 @@ __device__ __forceinline__ void filter_role(const RowArgs& a, const PipeCfg& cfg
     int it = 0;                // tiles this warp has filtered in this row
     bool overflow = false;
     // One tile: four pairs.  A pair is always stored at the cursor; the cursor moves on only for a hit,
-    // i.e. when max(pair) - thr has no sign bit.  A pair of NaNs counts as a hit and is dropped later; -inf
-    // never hits.
+    // i.e. when max(pair) >= thr.  A pair of NaNs and -inf never hit.
     auto filter_tile = [&](uint32_t ctile, uint32_t utile, float thr) {
       float y[8];
       tile_y8<DTYPE, HAS_U, HAS_T>(ctile, utile, lane, s2, t2, y);
@@ -484,13 +483,15 @@ __device__ __forceinline__ void filter_role(const RowArgs& a, const PipeCfg& cfg
         cur = list_base;
       }
       uint32_t d = cur;
+      imw <<= 4;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const float m = fmaxf(y[2 * k], y[2 * k + 1]);
-        const uint32_t miss = __umulhi(__float_as_uint(__fsub_rn(m, thr)), 2u);
         asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(d), "f"(y[2 * k]), "f"(y[2 * k + 1]) : "memory");
-        d = d + kStride - miss * kStride;
-        imw = imw * 2u + miss;
+        // hit: the cursor moves on; miss: the pair's bit is set in the inverted mask (both predicated, no branch)
+        asm("{\n\t.reg .pred p;\n\tsetp.ge.f32 p, %2, %3;\n\t@p add.u32 %0, %0, %4;\n\t@!p or.b32 %1, %1, %5;\n\t}"
+            : "+r"(d), "+r"(imw)
+            : "f"(m), "f"(thr), "r"(kStride), "r"(8u >> k));
       }
       cur = d;
       ++it;

@@ -40,6 +40,7 @@ class Workload:
     seed: int
     ragged_total: int = 0  # >0: window starts staggered uniformly in [0, ragged_total)
     prev_sigma: float = 0.5
+    row_spread: float = 0.0  # >0: row (b,i) is scaled by exp(row_spread * U(-1,1)): flat and peaked rows side by side
 
     @property
     def kcap(self) -> int:
@@ -82,6 +83,8 @@ def _sweep():
     out["v16k"] = base.scaled(name="v16k", V=16384, seed=302)
     out["v16k_f32"] = base.scaled(name="v16k_f32", V=16384, dtype=F32, seed=303)
     out["f16"] = base.scaled(name="f16", dtype=F16, seed=304)
+    # rows of very different sharpness in one batch (scale factors from 1/e to e), as a model's rows are
+    out["hetero"] = base.scaled(name="hetero", row_spread=1.0, seed=305)
     return out
 
 
@@ -133,6 +136,8 @@ def make_step_inputs(wl: Workload) -> StepInputs:
     rng = np.random.Generator(np.random.Philox(wl.seed))
     shape = (wl.B, wl.W, wl.V)
     cond = rng.standard_normal(shape, dtype=np.float32) * np.float32(wl.sigma)
+    if wl.row_spread > 0:
+        cond *= np.exp(wl.row_spread * rng.uniform(-1.0, 1.0, size=(wl.B, wl.W, 1))).astype(np.float32)
     if wl.peaks > 0:
         # `peaks` distinct ids per row, uniformly chosen, boosted by `boost`
         for b in range(wl.B):

@@ -9,7 +9,7 @@ from paper_2512_07503_b200 import workloads as wk
 pytestmark = pytest.mark.gpu
 
 CASES = [("w16", 6), ("w32", 4), ("w96", 2), ("w250", 1), ("w512", 1), ("k1", 2), ("k10", 2), ("k100", 2), ("k500", 2),
-         ("k1000", 2), ("k8192", 1), ("v32k", 3), ("v16k", 4), ("v16k_f32", 4), ("f16", 3)]
+         ("k1000", 2), ("k8192", 1), ("v32k", 3), ("v16k", 4), ("v16k_f32", 4), ("f16", 3), ("hetero", 4)]
 
 
 @pytest.mark.parametrize("name,B", CASES)
