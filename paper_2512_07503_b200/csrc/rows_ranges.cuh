@@ -1,18 +1,28 @@
 // Row kernel with one contiguous range of token ids per filter thread.
 //
-// Same three roles per CTA as rows_pipeline_kernel (producer / filter / finisher, one persistent CTA per
-// SM) and the same arithmetic; what differs is how a row is cut up.  The row of V logits is viewed as a
-// matrix of 256 ranges x R ids (R = V/256): filter thread t owns ids [t R, (t+1) R).  A ring stage is a
-// column slice of that matrix, 64 bytes per range, fetched by ONE tiled TMA copy per logits array
-// (cp.async.bulk.tensor, box {64 bytes, 256 ranges, 1 row}, 64-byte swizzle so that the 16-byte reads of
-// neighbouring threads fall into different banks).  Consequences:
+// One persistent CTA per SM, rows round-robin, four roles:
 //
-//   * stage 0 of a row is a systematic sample of it (64 bytes out of every R elements), so the sampling
-//     needs no schedule of its own;
+//   producer (1 warp)   streams rows through a ring of shared-memory stages with tiled TMA copies.
+//   sampler (4 warps)   works one row AHEAD of the filter: it gets a copy of the next row's stage 0 (a
+//                       systematic sample of that row) through the ring, and turns it into the candidate
+//                       threshold tau0 of that row while the filter warps are still streaming the current one.
+//   filter (8 warps)    merges the staged pairs into logits y and keeps the pairs that reach tau0; at the end
+//                       of the row it compacts its lists into a dense candidate list in ascending id order.
+//   finisher (8 warps)  one row BEHIND the filter: exact K-th largest among the candidates, softmax, output,
+//                       the row's own draw.
+//
+// The row of V logits is viewed as a matrix of 256 ranges x R ids (R = V/256): filter thread t owns ids
+// [t R, (t+1) R).  A ring stage is a column slice of that matrix, 64 bytes per range, fetched by ONE tiled
+// TMA copy per logits array (cp.async.bulk.tensor, box {64 bytes, 256 ranges, 1 row}, 64-byte swizzle so
+// that the 16-byte reads of neighbouring threads fall into different banks).  Consequences:
+//
+//   * stage 0 of a row is a systematic sample of it (64 bytes out of every R elements).  It is fetched
+//     twice: once a row early for the sampler, once in its turn for the filter (by then it sits in L2).
+//     Plain loads would not do for the sampler: behind the ring's outstanding copies they take thousands
+//     of cycles each;
 //   * a thread meets its ids in ascending order and thread t's ids all precede thread t+1's: the hit bits
 //     give the ids directly (id = t R + 2 * pair index) and the concatenation of the threads' lists IS the
-//     ascending-id order.  The finisher therefore needs no bitmap, no prefix over it and no scatter: it
-//     compacts the lists once, finds the exact K-th largest, and emits the survivors in list order.
+//     ascending-id order.  The finisher therefore needs no bitmap, no prefix over it and no scatter.
 //
 // Shapes: V = 256 R with R a multiple of the stage width (32 bf16 / 16 fp32 elements) and 2..16 stages per
 // row, rows at one uniform pitch.  Everything else goes to rows_pipeline_kernel or rows_generic_kernel.
@@ -24,74 +34,125 @@
 
 namespace sjd {
 
+// Phase timers: with -DSJD_PHASE_TIMERS thread 0 of every role adds the clock cycles between two marks to a
+// device-side table (read by sjd_phase_cycles_read); without it the marks compile to nothing.
+#ifdef SJD_PHASE_TIMERS
+__device__ unsigned long long g_phase_cycles[48];
+#define SJD_PHASE_BEGIN() long long phase_t0_ = clock64()
+#define SJD_PHASE(i)                                                                   \
+  do {                                                                                 \
+    if (tid == 0) {                                                                    \
+      const long long phase_t_ = clock64();                                            \
+      atomicAdd(&g_phase_cycles[i], (unsigned long long)(phase_t_ - phase_t0_));       \
+      phase_t0_ = phase_t_;                                                            \
+    }                                                                                  \
+  } while (0)
+#define SJD_PHASE_COUNT(i, n) \
+  do {                        \
+    if (tid == 0) atomicAdd(&g_phase_cycles[i], (unsigned long long)(n)); \
+  } while (0)
+#else
+#define SJD_PHASE_BEGIN()
+#define SJD_PHASE(i)
+#define SJD_PHASE_COUNT(i, n)
+#endif
+
 constexpr int kRangeThreads = 256;          // filter threads = ranges per row
 constexpr int kRangeStageBytes = 16384;     // one logits array in a ring stage: 64 bytes x 256 ranges
 constexpr int kRangeRingStages = 3;
-constexpr int kRangeDenseCap = 3584;        // candidates the finisher can hold for a row
+constexpr int kRangeListCap = 35;           // pair entries per filter thread and row (the last four are slack for
+                                            // the unconditional stores of one group)
+constexpr int kRangePairCap = 3328;         // candidate pairs the finisher can hold for a row
+constexpr int kPairChunk = (kRangePairCap + kRangeThreads - 1) / kRangeThreads;  // pairs per finisher thread
+constexpr int kSampleBins = 1024;           // sampler's histogram (group maxima by key, then linear bins)
+constexpr int kSampleKeyShift = 22;         // key bits dropped by the first histogram: sign, exponent, one mantissa bit
+constexpr int kRowsPerCta = 32;             // live rows a CTA takes in one launch (the host splits larger problems)
 
 struct RangeCfg {
   int sample_rank;  // m: rank (from the top) within the sample (stage 0) that fixes tau0
   int sample_all;   // 1: the first pass bins every sample element (m exceeds the number of groups of eight)
+  int group_rank;   // > 0: tau0 is the group maximum of this rank (the element rank m translated, see the sampler)
   int stages;       // S = R / (elements per stage and range)
   int range_len;    // R
   int mask_words;   // 32 hit bits each: R/2 pairs per range
+  int row_begin;    // this launch covers rows [row_begin, row_end)
+  int row_end;
 };
 
 enum {
   kRcAbort = 0,
-  kRcFBin, kRcFAbove, kRcFCount, kRcSmaxKey,          // filter
-  kRcRowTau0, kRcRowVmax, kRcRowTotal, kRcRowFallback,  // handed over with the row
+  kRcLive,                                              // live rows of this CTA (entries of the row table)
+  kRcABin, kRcAAbove, kRcACount, kRcSmaxKey,           // sampler
+  kRcTau0, kRcTau1, kRcTau2, kRcTau3,                   // tau0 of live row k in word kRcTau0 + (k & 3)
+  kRcTop0, kRcTop1, kRcTop2, kRcTop3,                   // largest sample value of live row k, likewise
+  kRcRowTau0, kRcRowTop, kRcRowPairs, kRcRowFallback,   // handed over with the row
   kRcPBin, kRcPAbove, kRcPCount, kRcGather, kRcPtok, kRcFoundId, kRcFoundP,  // finisher
-  kRcWords = 20
+  kRcWords = 32
 };
 
-struct BinMember {  // member of the threshold bin: value and where it sits in the dense list
+struct BinMember {  // member of the threshold bin: value and where it sits in the pair list (2 * pair + half)
   float y;
   int32_t slot;
 };
 
+struct RowEntry {  // one live row of this CTA with what the roles need to know about it
+  int32_t row;    // b * W + i
+  int32_t pos;    // absolute position of the row: pos_base[b] + i
+  int32_t iter;   // iteration counter of its sequence
+  int32_t draft;  // its draft token, -1 when every row is drafted
+};
+
 struct RangeSmem {
   unsigned char* ring;  // [kRangeRingStages][2][kRangeStageBytes], 1024-byte aligned
-  uint64_t* ylist;      // [kListCap][256] pair entries, one column per filter thread
+  uint64_t* ylist;      // [kRangeListCap][256] pair entries, one column per filter thread
   uint32_t* masks;      // [mask_words][256] inverted hit bits, first pair in the top bit
-  Candidate* dense;     // [kRangeDenseCap] candidates in ascending id order
+  uint64_t* pair_y;     // [kRangePairCap] candidate pairs {y(2q), y(2q+1)} in ascending id order
+  uint16_t* pair_q;     // [kRangePairCap] their pair numbers q (ids 2q and 2q+1)
   int32_t* st_ids;      // [kKcapMax] survivors, ascending id
   float* st_vals;       // [kKcapMax]
   uint32_t* sel;        // [kSelBins]  = st_ids: dead before the survivors are staged
   BinMember* binlist;   // [kBinListCap] = st_vals: likewise
-  uint32_t* hist;       // [kHistBins] filter
-  uint64_t* full;       // [kRangeRingStages]
-  uint64_t* empty;      // [kRangeRingStages]
+  uint32_t* hist;       // [kSampleBins] sampler
+  RowEntry* tab;        // [kRowsPerCta]
+  uint64_t* full;       // [kRangeRingStages] a row stage has landed in the slot (waited for by the filter)
+  uint64_t* empty;      // [kRangeRingStages] the slot's eight consumer warps are done with it
+  uint64_t* sample_full;  // [2] a sample has landed in its slot (row parity; waited for by the sampler)
+  uint64_t* tau_full;   // [2] tau0 of a row published by the sampler (row parity)
   uint64_t* cand_full;
   uint64_t* cand_free;
   uint64_t* scan_f;
   uint64_t* scan_p;
+  uint64_t* scan_a;
   int* ctl;
 };
 
 __host__ __device__ inline size_t range_smem_bytes(int mask_words) {
   size_t b = 1024;  // alignment slack for the swizzled ring
   b += (size_t)kRangeRingStages * 2 * kRangeStageBytes;
-  b += (size_t)kListCap * kRangeThreads * 8;
+  b += (size_t)kRangeListCap * kRangeThreads * 8;
   b += (size_t)mask_words * kRangeThreads * 4;
-  b += (size_t)kRangeDenseCap * sizeof(Candidate);
+  b += (size_t)kRangePairCap * (8 + 2);
   b += (size_t)kKcapMax * 8;
-  b += (size_t)kHistBins * 4;
-  b += 16 * 8 + 2 * (2 * 32 + 8) * 8 + kRcWords * 4;
+  b += (size_t)kSampleBins * 4;
+  b += (size_t)kRowsPerCta * sizeof(RowEntry);
+  b += 16 * 8 + 3 * (2 * 32 + 8) * 8 + kRcWords * 4;
   return b;
 }
 
 __device__ __forceinline__ RangeSmem carve_range_smem(unsigned char* base, int mask_words) {
   static_assert(sizeof(uint32_t) * kSelBins <= sizeof(int32_t) * kKcapMax, "sel must fit under st_ids");
   static_assert(sizeof(BinMember) * kBinListCap <= sizeof(float) * kKcapMax, "binlist must fit under st_vals");
+  static_assert((kRangePairCap * 2) % 16 == 0, "what follows the pair numbers stays 16-byte aligned");
   RangeSmem s;
   unsigned char* p = base + ((1024u - (smem_u32(base) & 1023u)) & 1023u);
   s.ring = p;
   p += (size_t)kRangeRingStages * 2 * kRangeStageBytes;
   s.ylist = reinterpret_cast<uint64_t*>(p);
-  p += (size_t)kListCap * kRangeThreads * 8;
-  s.dense = reinterpret_cast<Candidate*>(p);
-  p += (size_t)kRangeDenseCap * sizeof(Candidate);
+  p += (size_t)kRangeListCap * kRangeThreads * 8;
+  s.pair_y = reinterpret_cast<uint64_t*>(p);
+  p += (size_t)kRangePairCap * 8;
+  s.pair_q = reinterpret_cast<uint16_t*>(p);
+  p += (size_t)kRangePairCap * 2;
   s.st_ids = reinterpret_cast<int32_t*>(p);
   s.sel = reinterpret_cast<uint32_t*>(p);
   p += (size_t)kKcapMax * 4;
@@ -99,20 +160,76 @@ __device__ __forceinline__ RangeSmem carve_range_smem(unsigned char* base, int m
   s.binlist = reinterpret_cast<BinMember*>(p);
   p += (size_t)kKcapMax * 4;
   s.hist = reinterpret_cast<uint32_t*>(p);
-  p += (size_t)kHistBins * 4;
+  p += (size_t)kSampleBins * 4;
   s.masks = reinterpret_cast<uint32_t*>(p);
   p += (size_t)mask_words * kRangeThreads * 4;
+  s.tab = reinterpret_cast<RowEntry*>(p);
+  p += (size_t)kRowsPerCta * sizeof(RowEntry);
   s.full = reinterpret_cast<uint64_t*>(p);
   s.empty = s.full + kRangeRingStages;
-  s.cand_full = s.empty + kRangeRingStages;
+  s.sample_full = s.empty + kRangeRingStages;
+  s.tau_full = s.sample_full + 2;
+  s.cand_full = s.tau_full + 2;
   s.cand_free = s.cand_full + 1;
   p += 16 * 8;
   s.scan_f = reinterpret_cast<uint64_t*>(p);
   p += (2 * 32 + 8) * 8;
   s.scan_p = reinterpret_cast<uint64_t*>(p);
   p += (2 * 32 + 8) * 8;
+  s.scan_a = reinterpret_cast<uint64_t*>(p);
+  p += (2 * 32 + 8) * 8;
   s.ctl = reinterpret_cast<int*>(p);
   return s;
+}
+
+// Position in the ring of the CTA's n-th copy (the producer and both consumer groups count the same
+// sequence of copies): slot n mod NS, used for the (n / NS)-th time.  The sequence: the sample (stage 0) of
+// the first live row; then for every live row the sample of the next live row (if there is one) followed
+// by the row's own stages 0..S-1.  A slot's `empty` barrier sees every copy that goes through the slot, in
+// order, and only the producer waits on it.  Its `full` barrier completes for row stages only and the two
+// `sample_full` barriers for samples only, so that each is waited on by ONE group that takes its phases in
+// order: a parity wait tells a phase only from its neighbours, and a group waiting on a barrier that also
+// completes for the other group's copies would take one of those for its own.
+struct RingPos {
+  int slot;
+  uint32_t use;
+  __device__ __forceinline__ void step() {
+    if (++slot == kRangeRingStages) {
+      slot = 0;
+      ++use;
+    }
+  }
+  __device__ __forceinline__ void skip(int n) {
+    for (int j = 0; j < n; ++j) step();
+  }
+};
+
+// try_wait that may stay suspended in hardware for up to about `ns` nanoseconds before it reports "not yet"
+// (it returns at once when the phase completes): a waiting warp then spends next to no issue slots on polling.
+__device__ __forceinline__ bool mbar_try_wait_for(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait that also gives up when another role of the CTA has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait_abortable(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait_for(bar, parity, 4000u)) return true;
+    if ((i & 7u) == 7u) {
+      if (*abort_flag != 0) break;
+      if (clock64() - t0 > kSpinCycles) break;
+    }
+  }
+  return false;
 }
 
 // One tiled copy global -> shared: box {stage width, 256 ranges, 1 row} at element x of every range of
@@ -126,34 +243,15 @@ __device__ __forceinline__ void tma_load_box(void* dst, const CUtensorMap* map, 
 }
 
 // ---------------------------------------------------------------------------------------------------
-// filter warps
+// what the three consumer roles share: how a thread finds its 64 bytes of a staged slice
 // ---------------------------------------------------------------------------------------------------
-template <int DTYPE, bool HAS_U, bool HAS_T>
-__device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeCfg& cfg, const RangeSmem& sm, int tid) {
-  constexpr int NT_F = kRangeThreads;
-  constexpr int BAR_F = 1;
-  constexpr uint32_t kStride = NT_F * 8;         // bytes between consecutive entries of one filter thread
-  constexpr int TI = DTYPE != 0 ? 4 : 2;          // groups of eight elements per stage and thread
-  constexpr int NS = kRangeRingStages;
-  const int lane = tid & 31;
-  const int mask_words = cfg.mask_words;
-  const int rows = a.B * a.W;
-  const float neg_inf = __int_as_float(0xff800000);
-  const float lowest = -3.402823466e38f;  // with this threshold every finite value is a candidate
-  volatile int* abort_flag = sm.ctl + kRcAbort;
-  const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
-  const uint32_t ring_addr = smem_u32(sm.ring);
-  const uint32_t my_row = (uint32_t)tid * 64u;           // this thread's 64 bytes inside a staged array
-  const uint32_t swz = ((uint32_t)tid >> 1) & 3u;        // 64-byte swizzle: 16-byte piece j sits at j ^ swz
-  const uint32_t list_base = smem_u32(sm.ylist) + (uint32_t)tid * 8u;
-  const uint32_t list_limit = list_base + (uint32_t)(kListCap - 4) * kStride;  // beyond it a group may not fit
-  int slot = 0, flip = 0;
-  uint32_t phase = 0;
-  uint32_t n_row = 0;
-  bool dead = false;
-
+template <int DTYPE, bool HAS_U>
+struct StageReader {
+  uint32_t my_row;  // this thread's 64 bytes inside a staged array
+  uint32_t swz;     // 64-byte swizzle: 16-byte piece j sits at j ^ swz
+  __device__ __forceinline__ explicit StageReader(int tid) : my_row((uint32_t)tid * 64u), swz(((uint32_t)tid >> 1) & 3u) {}
   // the j-th group of eight elements of this thread in the staged slice at `stage`
-  auto load_group = [&](uint32_t stage, int j, RawTile<DTYPE>& r) {
+  __device__ __forceinline__ void load_group(uint32_t stage, int j, RawTile<DTYPE>& r) const {
     if (DTYPE != 0) {
       r.c[0] = lds128(stage + my_row + (((uint32_t)j ^ swz) << 4));
       if (HAS_U) r.u[0] = lds128(stage + kRangeStageBytes + my_row + (((uint32_t)j ^ swz) << 4));
@@ -165,54 +263,188 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
         r.u[DTYPE != 0 ? 0 : 1] = lds128(stage + kRangeStageBytes + my_row + (((uint32_t)(2 * j + 1) ^ swz) << 4));
       }
     }
-  };
+  }
+};
 
-  for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-    // from the block's last row on, the verification grid may be scheduled (it waits for this grid's end)
-    if (row + (int)gridDim.x >= rows) allow_dependent_launch();
-    const int b = row / a.W, i = row - b * a.W;
-    const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
-    if (i >= L || dead) continue;
-
-    // ---------------- stage 0 is the sample.  First pass: maxima of groups of eight, by key ----------------
-    bool ok = mbar_wait(&sm.full[slot], phase);
+// ---------------------------------------------------------------------------------------------------
+// sampler warps: tau0 of the NEXT row from its stage 0, while the filter warps stream the current row
+// ---------------------------------------------------------------------------------------------------
+// Threshold in two steps: maxima of groups of eight -> histogram by order-preserving key -> floor f with
+// enough group maxima above it; linear histogram over [f, sample max] -> tau0.  Two ways through the second
+// step:
+//   * by group maxima (group_rank > 0, the usual case: the wanted rank m is a small fraction p = m / n of the
+//     sample): with exchangeable entries a group of eight has its maximum above t with probability
+//     1 - (1 - p(t))^8, so the value whose rank among the group maxima is g = n/8 (1 - (1 - p)^8) has rank m
+//     among the elements on average.  Only the eight maxima a thread holds are binned again;
+//   * by elements (group_rank == 0): the sample stays in registers as packed half-precision values between
+//     the two steps and every value above f is binned.
+// Either way the ring slot is given back as soon as the sample is in registers.  tau0 only steers how many
+// candidates the filter keeps (the result is exact whatever it is; too few candidates send the row to the
+// any-shape path), so neither the rounding to 11 bits nor the translation of the rank costs exactness.
+// Sampler thread t looks after ranges t and t + 128.
+template <int DTYPE, bool HAS_U, bool HAS_T, bool BY_GROUPS, int NA>
+__device__ __forceinline__ void range_sampler_role(const RowArgs& a, const RangeCfg& cfg, const RangeSmem& sm, int tid) {
+  constexpr int NT_A = NA * 32;
+  constexpr int BAR_A = 3;
+  constexpr int TI = DTYPE != 0 ? 4 : 2;        // groups of eight elements per range in stage 0
+  constexpr int NR = kRangeThreads / NT_A;       // ranges per sampler thread
+  constexpr int NG = NR * TI;                    // groups per sampler thread
+  static_assert(kRangeThreads % NT_A == 0, "ranges must split evenly over the sampler threads");
+  const int lane = tid & 31;
+  const float neg_inf = __int_as_float(0xff800000);
+  const float lowest = -3.402823466e38f;  // with this threshold every finite value is a candidate
+  volatile int* abort_flag = sm.ctl + kRcAbort;
+  const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
+  const uint32_t ring_addr = smem_u32(sm.ring);
+  const uint32_t n_live = (uint32_t)sm.ctl[kRcLive];
+  RingPos pos{0, 0};
+  int flip = 0;
+  for (uint32_t k = 0; k < n_live; ++k) {  // live rows of this CTA
+    SJD_PHASE_BEGIN();
+    // ---------------- the sample into registers; first pass on the way: maxima of groups of eight, by key ----------------
+    const bool ok = mbar_wait_abortable(&sm.sample_full[k & 1u], (k >> 1) & 1u, abort_flag);
+    SJD_PHASE(0);
+    __half2 cache[BY_GROUPS ? 1 : NG * 4];
+    float gmax[NG];
     float smax = neg_inf;
-    const uint32_t stage0 = ring_addr + (uint32_t)slot * (2 * kRangeStageBytes);
+    constexpr bool by_groups = BY_GROUPS;
+    const uint32_t rank = (uint32_t)(by_groups ? cfg.group_rank : cfg.sample_rank);
+#pragma unroll
+    for (int g = 0; g < NG; ++g) gmax[g] = neg_inf;
     if (ok) {
+      const uint32_t stage0 = ring_addr + (uint32_t)pos.slot * (2 * kRangeStageBytes);
 #pragma unroll
-      for (int j = 0; j < TI; ++j) {
-        RawTile<DTYPE> raw;
-        load_group(stage0, j, raw);
-        float y[8];
-        merge_raw<DTYPE, HAS_U, HAS_T>(raw, s2, t2, y);
-        const float m8 = max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]);
-        if (cfg.sample_all) {
+      for (int r = 0; r < NR; ++r) {
+        const StageReader<DTYPE, HAS_U> rd(tid + r * NT_A);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) atomicAdd(&sm.hist[float_key(canonical(y[k])) >> 21], 1u);
-        } else {
-          atomicAdd(&sm.hist[float_key(canonical(m8)) >> 21], 1u);
+        for (int j = 0; j < TI; ++j) {
+          RawTile<DTYPE> raw;
+          rd.load_group(stage0, j, raw);
+          float y[8];
+          merge_raw<DTYPE, HAS_U, HAS_T>(raw, s2, t2, y);
+          const float m8 = canonical(max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]));
+          gmax[r * TI + j] = m8;
+          if (!by_groups) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) y[q] = canonical(y[q]);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) cache[BY_GROUPS ? 0 : (r * TI + j) * 4 + q] = __floats2half2_rn(y[2 * q], y[2 * q + 1]);
+          }
+          if (!BY_GROUPS && cfg.sample_all) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) atomicAdd(&sm.hist[float_key(y[q]) >> kSampleKeyShift], 1u);
+          } else {
+            // group maxima crowd into a few coarse bins: one atomic per distinct bin of the warp
+            const uint32_t bin = float_key(m8) >> kSampleKeyShift;
+            const uint32_t peers = __match_any_sync(0xffffffffu, bin);
+            if ((peers & ((1u << lane) - 1u)) == 0u) atomicAdd(&sm.hist[bin], (uint32_t)__popc(peers));
+          }
+          smax = fmaxf(smax, m8);
         }
-        smax = fmaxf(smax, m8);
       }
     }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[pos.slot], 8 / NA);  // the slot's barrier counts eight warps
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, d));
-    if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(&sm.ctl[kRcSmaxKey]), float_key(canonical(smax)));
-    dead = group_any<NT_F, BAR_F>(!ok);
-    if (dead) {
+    if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(&sm.ctl[kRcSmaxKey]), float_key(smax));
+    if (group_any<NT_A, BAR_A>(!ok)) {
       if (tid == 0) *abort_flag = 1;
-      continue;
+      return;
     }
+    SJD_PHASE(1);
     // at least m group maxima (or, binning everything, m elements), hence at least m sample elements, are >=
     // the lower edge of this bin
-    find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kRcFBin);
-    const int cbin = sm.ctl[kRcFBin];
-    float floor_y = cbin >= 0 ? key_float((uint32_t)cbin << 21) : lowest;
+    find_rank_bin<kSampleBins, NT_A, BAR_A>(sm.hist, rank, tid, sm.scan_a, flip, sm.ctl, kRcABin);
+    SJD_PHASE(2);
+    const int cbin = sm.ctl[kRcABin];
+    float floor_y = cbin >= 0 ? key_float((uint32_t)cbin << kSampleKeyShift) : lowest;
     if (!(floor_y >= lowest)) floor_y = lowest;  // edge fell on -inf or into the NaN patterns
     const float top_y = key_float((uint32_t)sm.ctl[kRcSmaxKey]);
     const bool refine = floor_y > lowest && top_y >= floor_y && top_y <= 3.402823466e38f;
     const float range = __fsub_rn(top_y, floor_y);
-    const float scale = (refine && range > 0.0f) ? __fdiv_rn((float)kHistBins - 0.5f, range) : 0.0f;
+    const float scale = (refine && range > 0.0f) ? __fdiv_rn((float)kSampleBins - 0.5f, range) : 0.0f;
+    // ---------------- second pass: linear bins over [floor, sample max] ----------------
+    float tau0 = lowest;
+    if (refine) {
+      if (by_groups) {
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          const int bin = min(max(__float2int_rd(__fmul_rn(__fsub_rn(gmax[g], floor_y), scale)), 0), kSampleBins - 1);
+          if (gmax[g] >= floor_y) atomicAdd(&sm.hist[bin], 1u);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < (BY_GROUPS ? 0 : NG * 4); ++j) {
+          const float2 v = __half22float2(cache[j]);
+          const int b0 = min(max(__float2int_rd(__fmul_rn(__fsub_rn(v.x, floor_y), scale)), 0), kSampleBins - 1);
+          const int b1 = min(max(__float2int_rd(__fmul_rn(__fsub_rn(v.y, floor_y), scale)), 0), kSampleBins - 1);
+          if (v.x >= floor_y) atomicAdd(&sm.hist[b0], 1u);
+          if (v.y >= floor_y) atomicAdd(&sm.hist[b1], 1u);
+        }
+      }
+      group_sync<NT_A, BAR_A>();
+      SJD_PHASE(3);
+      if (tid == 0) sm.ctl[kRcSmaxKey] = 0;  // every thread has read it; next written after the next row's barriers
+      find_rank_bin<kSampleBins, NT_A, BAR_A>(sm.hist, rank, tid, sm.scan_a, flip, sm.ctl, kRcABin);
+      const int fbin = sm.ctl[kRcABin];
+      if (fbin > 0 && scale > 0.0f) {
+        // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
+        const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
+        tau0 = __fadd_rd(floor_y, t);
+      } else if (fbin >= 0) {
+        tau0 = floor_y;
+      }
+    } else {
+      group_sync<NT_A, BAR_A>();
+      if (tid == 0) sm.ctl[kRcSmaxKey] = 0;
+    }
+    // a word of its own for each of four consecutive rows: the filter reads it at the start of the row, and
+    // the ring keeps the sampler less than two rows ahead of the filter
+    if (tid == 0) {
+      sm.ctl[kRcTau0 + (int)(k & 3u)] = __float_as_int(tau0);
+      sm.ctl[kRcTop0 + (int)(k & 3u)] = __float_as_int(top_y);
+      mbar_arrive(&sm.tau_full[k & 1u]);
+    }
+    group_sync<NT_A, BAR_A>();  // kRcABin is rewritten by the next row's first search
+    SJD_PHASE(4);
+    // sample(1) follows sample(0) directly; sample(k+1) follows sample(k) after the S stages of row k-1 and itself
+    if (k == 0) pos.step();
+    else pos.skip(1 + cfg.stages);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// filter warps
+// ---------------------------------------------------------------------------------------------------
+template <int DTYPE, bool HAS_U, bool HAS_T>
+__device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeCfg& cfg, const RangeSmem& sm, int tid) {
+  constexpr int NT_F = kRangeThreads;
+  constexpr int BAR_F = 1;
+  constexpr uint32_t kStride = NT_F * 8;         // bytes between consecutive entries of one filter thread
+  constexpr int TI = DTYPE != 0 ? 4 : 2;          // groups of eight elements per stage and thread
+  const int lane = tid & 31;
+  const int mask_words = cfg.mask_words;
+  volatile int* abort_flag = sm.ctl + kRcAbort;
+  const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
+  const uint32_t ring_addr = smem_u32(sm.ring);
+  const StageReader<DTYPE, HAS_U> rd(tid);
+  const uint32_t list_base = smem_u32(sm.ylist) + (uint32_t)tid * 8u;
+  const uint32_t list_limit = list_base + (uint32_t)(kRangeListCap - 4) * kStride;  // beyond it a group may not fit
+  const uint32_t n_live = (uint32_t)sm.ctl[kRcLive];
+  RingPos pos{0, 0};
+  pos.step();  // the CTA's first copy is the first row's sample
+  uint32_t full_phase = 0;  // bit s: parity of the next phase of full[s] this group waits for
+  int flip = 0;
+  for (uint32_t k = 0; k < n_live; ++k) {  // live rows of this CTA
+    // from the CTA's last row on, the verification grid may be scheduled (it waits for this grid's end)
+    if (k + 1 == n_live) allow_dependent_launch();
+    else pos.step();  // the next row's sample comes before this row's stages
+    SJD_PHASE_BEGIN();
+    bool ok = mbar_wait_abortable(&sm.tau_full[k & 1u], (k >> 1) & 1u, abort_flag);
+    SJD_PHASE(8);
+    const float tau0 = __int_as_float(sm.ctl[kRcTau0 + (int)(k & 3u)]);
+    const int top_bits = sm.ctl[kRcTop0 + (int)(k & 3u)];
 
     uint32_t cur = list_base;  // shared-memory address of the thread's next free entry
     uint32_t imw = 0;          // inverted hit bits of the groups filtered since the last full mask word
@@ -229,13 +461,13 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
       uint32_t d = cur;
       imw <<= 4;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float m = fmaxf(y[2 * k], y[2 * k + 1]);
-        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(d), "f"(y[2 * k]), "f"(y[2 * k + 1]) : "memory");
+      for (int q = 0; q < 4; ++q) {
+        const float m = fmaxf(y[2 * q], y[2 * q + 1]);
+        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(d), "f"(y[2 * q]), "f"(y[2 * q + 1]) : "memory");
         // hit: the cursor moves on; miss: the pair's bit is set in the inverted mask (both predicated, no branch)
         asm("{\n\t.reg .pred p;\n\tsetp.ge.f32 p, %2, %3;\n\t@p add.u32 %0, %0, %4;\n\t@!p or.b32 %1, %1, %5;\n\t}"
             : "+r"(d), "+r"(imw)
-            : "f"(m), "f"(thr), "r"(kStride), "r"(8u >> k));
+            : "f"(m), "f"(thr), "r"(kStride), "r"(8u >> q));
       }
       cur = d;
     };
@@ -247,73 +479,28 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
         imw = 0;
       }
     };
-    // ---------------- the sample against the floor (a superset of what tau0 will keep) ----------------
-    const float sample_thr = refine ? floor_y : lowest;
-#pragma unroll
-    for (int j = 0; j < TI; ++j) {
-      RawTile<DTYPE> raw;
-      load_group(stage0, j, raw);
-      filter_group(raw, sample_thr);
-    }
-    end_stage(0);
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.empty[slot]);
-    if (++slot == NS) {
-      slot = 0;
-      phase ^= 1u;
-    }
-    // ---------------- second pass: linear bins over [floor, sample max], from the lists ----------------
-    float tau0 = lowest;
-    if (refine) {
-      for (uint32_t e = list_base; e < cur; e += kStride) {
-        float v0, v1;
-        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v0), "=f"(v1) : "r"(e));
-        if (v0 >= floor_y) {
-          const int q = __float2int_rd(__fmul_rn(__fsub_rn(v0, floor_y), scale));
-          atomicAdd(&sm.hist[min(max(q, 0), kHistBins - 1)], 1u);
-        }
-        if (v1 >= floor_y) {
-          const int q = __float2int_rd(__fmul_rn(__fsub_rn(v1, floor_y), scale));
-          atomicAdd(&sm.hist[min(max(q, 0), kHistBins - 1)], 1u);
-        }
-      }
-      group_sync<NT_F, BAR_F>();
-      if (tid == 0) sm.ctl[kRcSmaxKey] = 0;  // every thread has read it; next written after the next row's barriers
-      find_rank_bin<kHistBins, NT_F, BAR_F>(sm.hist, (uint32_t)cfg.sample_rank, tid, sm.scan_f, flip, sm.ctl, kRcFBin);
-      const int fbin = sm.ctl[kRcFBin];
-      if (fbin > 0 && scale > 0.0f) {
-        // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
-        const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
-        tau0 = __fadd_rd(floor_y, t);
-      } else if (fbin >= 0) {
-        tau0 = floor_y;
-      }
-    } else {
-      group_sync<NT_F, BAR_F>();
-      if (tid == 0) sm.ctl[kRcSmaxKey] = 0;
-    }
-    // ---------------- the rest of the row against tau0 ----------------
-    for (int s = 1; s < cfg.stages; ++s) {
-      if (ok) ok = mbar_wait(&sm.full[slot], phase);
+    // ---------------- the row against tau0 ----------------
+    for (int s = 0; s < cfg.stages; ++s) {
+      if (ok) ok = mbar_wait_abortable(&sm.full[pos.slot], (full_phase >> pos.slot) & 1u, abort_flag);
+      full_phase ^= 1u << pos.slot;
       if (ok) {
-        const uint32_t stage = ring_addr + (uint32_t)slot * (2 * kRangeStageBytes);
+        const uint32_t stage = ring_addr + (uint32_t)pos.slot * (2 * kRangeStageBytes);
         RawTile<DTYPE> raw[TI];
 #pragma unroll
-        for (int j = 0; j < TI; ++j) load_group(stage, j, raw[j]);
+        for (int j = 0; j < TI; ++j) rd.load_group(stage, j, raw[j]);
 #pragma unroll
         for (int j = 0; j < TI; ++j) filter_group(raw[j], tau0);
         end_stage(s);
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.empty[slot]);
-      if (++slot == NS) {
-        slot = 0;
-        phase ^= 1u;
-      }
+      if (lane == 0) mbar_arrive(&sm.empty[pos.slot]);
+      pos.step();
     }
-    // ---------------- drain: this thread's list becomes its run of the dense list ----------------
+    SJD_PHASE(9);
+    // ---------------- drain: this thread's list becomes its run of the pair list ----------------
     // Threads own ascending id ranges and meet their ids in ascending order, so writing the runs one
-    // after the other yields the candidates in ascending id order.
+    // after the other yields the candidate pairs in ascending id order.  A pair goes over as it is; the
+    // finisher sorts out which of its two values reach tau0.
     {
       const int it = cfg.stages * TI;  // groups of eight this thread has filtered in this row
       const int rem = it & 7;
@@ -326,149 +513,179 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
       for (; w < mask_words; ++w) sm.masks[(size_t)w * NT_F + tid] = 0xffffffffu;
     }
     const int n_e = overflow ? 0 : (int)((cur - list_base) / kStride);
-    uint32_t my_valid = 0;
-    float vmax = neg_inf;
-    for (int e = 0; e < n_e; ++e) {
-      float v0, v1;
-      asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v0), "=f"(v1) : "r"(list_base + (uint32_t)e * kStride));
-      if (v0 >= tau0) {
-        ++my_valid;
-        vmax = fmaxf(vmax, v0);
-      }
-      if (v1 >= tau0) {
-        ++my_valid;
-        vmax = fmaxf(vmax, v1);
-      }
-    }
-    uint32_t n_total;
-    uint32_t my_off = group_scan1<NT_F, BAR_F, uint32_t>(my_valid, tid, sm.scan_f, flip, &n_total);
-    vmax = group_max1_f32<NT_F, BAR_F>(vmax, tid, sm.scan_f, flip);
-    // the dense list must be back from the finisher
-    if (ok && n_row > 0) ok = mbar_wait(sm.cand_free, (n_row - 1) & 1u);
-    const bool any_overflow = group_any<NT_F, BAR_F>(overflow);
-    dead = group_any<NT_F, BAR_F>(!ok);
-    if (dead) {
+    // the pair list must be back from the finisher
+    if (ok && k > 0) ok = mbar_wait_abortable(sm.cand_free, (k - 1) & 1u, abort_flag);
+    SJD_PHASE(10);
+    // one scan carries the entry counts (bits 0-13: at most 35 each) and the number of threads whose list ran
+    // over (bits 14-22) or whose wait gave up (bits 23-31)
+    uint32_t sum;
+    const uint32_t mine = (uint32_t)n_e | (overflow ? 1u << 14 : 0u) | (ok ? 0u : 1u << 23);
+    const uint32_t my_off = group_scan1<NT_F, BAR_F, uint32_t>(mine, tid, sm.scan_f, flip, &sum) & 0x3fffu;
+    if ((sum >> 23) != 0u) {
       if (tid == 0) *abort_flag = 1;
-      continue;  // the row is not handed over: the finisher's wait runs out and marks the rows
+      return;  // the row is not handed over: the finisher's wait ends on the flag and it marks the rows
     }
-    // too few candidates (the sampled threshold was too high), too many for the list, or no finite maximum:
-    // the finisher redoes the row by the any-shape path
-    const bool fallback = any_overflow || n_total < (uint32_t)a.kcap || n_total > (uint32_t)kRangeDenseCap ||
-                          !(vmax <= 3.402823466e38f);
+    const uint32_t n_pairs = sum & 0x3fffu;
+    // a list that ran over, or more pairs than the finisher holds: it redoes the row by the any-shape path
+    const bool fallback = ((sum >> 14) & 0x1ffu) != 0u || n_pairs > (uint32_t)kRangePairCap;
+    SJD_PHASE(11);
     if (!fallback) {
-      const int id0 = tid * cfg.range_len;
-      int e = 0;
-      for (int w = 0; w < mask_words; ++w) {
-        uint32_t x = ~sm.masks[(size_t)w * NT_F + tid];
-        while (x != 0u && e < n_e) {
-          const int bitpos = __clz((int)x);
-          x &= ~(0x80000000u >> bitpos);
-          const int id = id0 + 2 * (w * 32 + bitpos);  // pair q of range t holds ids t R + 2q and t R + 2q + 1
-          float v0, v1;
-          asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v0), "=f"(v1) : "r"(list_base + (uint32_t)e * kStride));
-          ++e;
-          if (v0 >= tau0) sm.dense[my_off++] = Candidate{canonical(v0), id};
-          if (v1 >= tau0) sm.dense[my_off++] = Candidate{canonical(v1), id + 1};
+      const uint32_t q0 = (uint32_t)(tid * (cfg.range_len >> 1));  // first pair number of this thread's range
+      int w = 0;
+      uint32_t x = ~sm.masks[tid];
+      for (int e0 = 0; e0 < n_e; e0 += 4) {
+        uint64_t v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)  // entries past n_e are read (inside the list) and dropped
+          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v[u]) : "r"(list_base + (uint32_t)min(e0 + u, kRangeListCap - 1) * kStride));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (e0 + u < n_e) {
+            while (x == 0u && w + 1 < mask_words) {
+              ++w;
+              x = ~sm.masks[(size_t)w * NT_F + tid];
+            }
+            const int bitpos = __clz((int)x);
+            x &= ~(0x80000000u >> bitpos);
+            sm.pair_y[my_off + e0 + u] = v[u];
+            sm.pair_q[my_off + e0 + u] = (uint16_t)(q0 + (uint32_t)(w * 32 + bitpos));
+          }
         }
       }
     }
     group_sync<NT_F, BAR_F>();
     if (tid == 0) {
       sm.ctl[kRcRowTau0] = __float_as_int(tau0);
-      sm.ctl[kRcRowVmax] = __float_as_int(vmax);
-      sm.ctl[kRcRowTotal] = (int)n_total;
+      sm.ctl[kRcRowTop] = top_bits;
+      sm.ctl[kRcRowPairs] = (int)n_pairs;
       sm.ctl[kRcRowFallback] = fallback ? 1 : 0;
       mbar_arrive(sm.cand_full);
     }
-    ++n_row;
+    SJD_PHASE(12);
   }
+}
+
+// The any-shape path for a row the single pass could not finish: rare, so kept out of line (the finisher's
+// code stays small).  Its scratch sits on st_vals, so that the bins (= st_ids) stay clear.
+template <int DTYPE, int NT, int BAR>
+__device__ __noinline__ void redo_row(const RowArgs& a, int row, int tid, float* st_vals) {
+  row_generic<DTYPE, NT, BAR>(a, row, tid, *reinterpret_cast<GenericSmem*>(st_vals), kRowStatusRedone);
 }
 
 // ---------------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------------
-template <int DTYPE, int NP>
-__global__ void __launch_bounds__((8 + NP + 1) * 32, 1)
+template <int DTYPE, int NP, int NA>
+__global__ void __launch_bounds__((8 + NP + NA + 1) * 32, 1)
 rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ CUtensorMap map_c,
                    const __grid_constant__ CUtensorMap map_u) {
   constexpr int NF = 8;
   constexpr int NT_F = kRangeThreads, NT_P = NP * 32;
-  constexpr int BAR_P = 2;  // named barrier of the finisher warps (the filter warps use 1)
+  constexpr int BAR_P = 2;  // named barrier of the finisher warps (the filter warps use 1, the sampler warps 3)
   constexpr int kFinItems = kKcapMax / NT_P;
   constexpr int NS = kRangeRingStages;
   constexpr int BW = 64 / (DTYPE != 0 ? 2 : 4);  // elements per stage and range
-  static_assert(NT_F == NF * 32 && kFinItems == 8, "group sizes");
+  static_assert(NT_F == NF * 32 && NT_P == kRangeThreads && kFinItems == 8, "group sizes");
   extern __shared__ unsigned char smem_raw[];
   RangeSmem sm = carve_range_smem(smem_raw, cfg.mask_words);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool has_u = a.uncond != nullptr;
   const float neg_inf = __int_as_float(0xff800000);
-  const int rows = a.B * a.W;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(&sm.full[s], 1);
       mbar_init(&sm.empty[s], NF);
     }
+    for (int p = 0; p < 2; ++p) {
+      mbar_init(&sm.sample_full[p], 1);
+      mbar_init(&sm.tau_full[p], 1);
+    }
     mbar_init(sm.cand_full, 1);
     mbar_init(sm.cand_free, 1);
     for (int k = 0; k < kRcWords; ++k) sm.ctl[k] = 0;
     fence_barrier_init();
   }
-  for (int j = threadIdx.x; j < kHistBins; j += blockDim.x) sm.hist[j] = 0;
+  for (int j = threadIdx.x; j < kSampleBins; j += blockDim.x) sm.hist[j] = 0;
   for (int j = threadIdx.x; j < kSelBins; j += blockDim.x) sm.sel[j] = 0;
   // everything above touched shared memory only; global memory is read and written from here on, so a
   // launch that was allowed to overlap the previous kernel of the stream waits for that kernel's end here
   grid_dependency_wait();
   __syncthreads();
-  volatile int* abort_flag = sm.ctl + kRcAbort;
-
-  if (warp == NF + NP) {
-    // ====================================== producer warp ======================================
-    if (lane != 0) return;
-    int slot = 0;
-    uint32_t use = 0, issued = 0;
-    bool ok = true;
-    const uint32_t stage_bytes = (uint32_t)kRangeStageBytes * (has_u ? 2u : 1u);
-    for (int row = blockIdx.x; row < rows && ok; row += gridDim.x) {
+  // ---- the CTA's rows: row_begin + blockIdx.x, + gridDim.x, ... (at most kRowsPerCta of them inside
+  // [row_begin, row_end), which the host guarantees).  Rows beyond their sequence's window length have no
+  // logits to look at and get their empty result here; the others go into a table with everything the roles
+  // need to know about them, so that no role reads global memory at a row boundary (behind the ring's
+  // outstanding copies such a load takes thousands of cycles).
+  if (warp == 0) {
+    const int row = cfg.row_begin + (int)blockIdx.x + lane * (int)gridDim.x;
+    bool live = false;
+    RowEntry e{row, 0, 0, -1};
+    if (row < cfg.row_end) {
       const int b = row / a.W, i = row - b * a.W;
       const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
-      if (i >= L) continue;
-      for (int s = 0; s < cfg.stages; ++s) {
-        if (use > 0) ok = mbar_wait(&sm.empty[slot], (use - 1) & 1u);
-        ok = ok && (*abort_flag == 0);
-        if (!ok) break;
-        unsigned char* dst = sm.ring + (size_t)slot * (2 * kRangeStageBytes);
-        mbar_arrive_expect_tx(&sm.full[slot], stage_bytes);
-        tma_load_box(dst, &map_c, s * BW, row, &sm.full[slot]);
-        if (has_u) tma_load_box(dst + kRangeStageBytes, &map_u, s * BW, row, &sm.full[slot]);
-        ++issued;
-        if (++slot == NS) {
-          slot = 0;
-          ++use;
-        }
+      live = i < L;
+      if (live) {
+        e.pos = (a.pos_base ? a.pos_base[b] : 0) + i;
+        e.iter = a.iteration ? a.iteration[b] : a.iteration0;
+        e.draft = a.drafts ? a.drafts[row] : -1;
+      } else {
+        a.out_cnt[row] = 0;
+        a.scratch[row] = RowScratch{0.0f, -1, 0.0f, 0};
       }
     }
-    // drain: every stage armed here must have landed before the CTA may exit
-    {
-      const uint32_t n_back = issued < (uint32_t)NS ? issued : (uint32_t)NS;
-      int sl = slot;
-      uint32_t us = use;
-      for (uint32_t k = 0; k < n_back; ++k) {
-        if (--sl < 0) {
-          sl = NS - 1;
-          --us;
-        }
-        mbar_wait(&sm.full[sl], us & 1u);
+    const uint32_t votes = __ballot_sync(0xffffffffu, live);
+    if (live) sm.tab[__popc(votes & ((1u << lane) - 1u))] = e;
+    if (lane == 0) sm.ctl[kRcLive] = __popc(votes);
+  }
+  __syncthreads();
+  volatile int* abort_flag = sm.ctl + kRcAbort;
+  const int n_live = sm.ctl[kRcLive];
+
+  if (warp == NF + NP + NA) {
+    // ====================================== producer warp ======================================
+    if (lane != 0) return;
+    RingPos pos{0, 0};
+    bool ok = true;
+    const uint32_t stage_bytes = (uint32_t)kRangeStageBytes * (has_u ? 2u : 1u);
+    uint64_t* last_bar[NS] = {};  // barrier the latest copy into each slot completes on
+    uint32_t last_parity[NS] = {};
+    uint32_t n_stage_copies[NS] = {};  // row stages that have gone through each slot
+    auto issue = [&](int x, int row, int sample_of) {  // sample_of: -1 for a row stage, else the live row's index
+      if (pos.use > 0) ok = mbar_wait_abortable(&sm.empty[pos.slot], (pos.use - 1) & 1u, abort_flag);
+      ok = ok && (*abort_flag == 0);
+      if (!ok) return;
+      unsigned char* dst = sm.ring + (size_t)pos.slot * (2 * kRangeStageBytes);
+      uint64_t* bar;
+      if (sample_of >= 0) {
+        bar = &sm.sample_full[sample_of & 1];
+        last_parity[pos.slot] = ((uint32_t)sample_of >> 1) & 1u;
+      } else {
+        bar = &sm.full[pos.slot];
+        last_parity[pos.slot] = n_stage_copies[pos.slot]++ & 1u;
       }
-      if (!ok) *abort_flag = 1;
+      last_bar[pos.slot] = bar;
+      mbar_arrive_expect_tx(bar, stage_bytes);
+      tma_load_box(dst, &map_c, x, row, bar);
+      if (has_u) tma_load_box(dst + kRangeStageBytes, &map_u, x, row, bar);
+      pos.step();
+    };
+    if (n_live > 0) issue(0, sm.tab[0].row, 0);
+    for (int k = 0; k < n_live && ok; ++k) {
+      if (k + 1 < n_live) issue(0, sm.tab[k + 1].row, k + 1);
+      const int row = sm.tab[k].row;
+      for (int s = 0; s < cfg.stages && ok; ++s) issue(s * BW, row, -1);
     }
+    // drain: every copy armed here must have landed before the CTA may exit
+    for (int sl = 0; sl < NS; ++sl)
+      if (last_bar[sl] != nullptr) mbar_wait(last_bar[sl], last_parity[sl]);
+    if (!ok) *abort_flag = 1;
     return;
   }
 
+  const bool has_t = a.inv_T != 1.0f;
   if (warp < NF) {
     // ======================================= filter warps =======================================
-    const bool has_t = a.inv_T != 1.0f;
     if (has_u) {
       if (has_t) range_filter_role<DTYPE, true, true>(a, cfg, sm, threadIdx.x);
       else range_filter_role<DTYPE, true, false>(a, cfg, sm, threadIdx.x);
@@ -478,33 +695,47 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     }
     return;
   }
+  if (warp >= NF + NP) {
+    // ======================================= sampler warps =======================================
+    const int t = threadIdx.x - (NF + NP) * 32;
+    if (cfg.group_rank > 0) {
+      if (has_u) {
+        if (has_t) range_sampler_role<DTYPE, true, true, true, NA>(a, cfg, sm, t);
+        else range_sampler_role<DTYPE, true, false, true, NA>(a, cfg, sm, t);
+      } else {
+        if (has_t) range_sampler_role<DTYPE, false, true, true, NA>(a, cfg, sm, t);
+        else range_sampler_role<DTYPE, false, false, true, NA>(a, cfg, sm, t);
+      }
+    } else {
+      if (has_u) {
+        if (has_t) range_sampler_role<DTYPE, true, true, false, NA>(a, cfg, sm, t);
+        else range_sampler_role<DTYPE, true, false, false, NA>(a, cfg, sm, t);
+      } else {
+        if (has_t) range_sampler_role<DTYPE, false, true, false, NA>(a, cfg, sm, t);
+        else range_sampler_role<DTYPE, false, false, false, NA>(a, cfg, sm, t);
+      }
+    }
+    return;
+  }
 
   // ======================================= finisher warps =======================================
-  const int tid = threadIdx.x - NT_F;  // 0 .. NT_P-1; also the filter thread whose list this thread drains
+  const int tid = threadIdx.x - NT_F;  // 0 .. NT_P-1
   int flip = 0;
-  uint32_t n_row = 0;
   bool dead = false;
-  for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-    // from the block's last row on, the verification grid may be scheduled (it waits for this grid's end)
-    if (row + (int)gridDim.x >= rows) allow_dependent_launch();
-    const int b = row / a.W, i = row - b * a.W;
-    const int L = a.win_len ? min(max(a.win_len[b], 0), a.W) : a.W;
+  float* const pair_vals = reinterpret_cast<float*>(sm.pair_y);  // value 2p + h is half h of pair p
+  for (int k = 0; k < n_live; ++k) {
+    // from the CTA's last row on, the verification grid may be scheduled (it waits for this grid's end)
+    if (k + 1 == n_live) allow_dependent_launch();
+    SJD_PHASE_BEGIN();
+    const RowEntry re = sm.tab[k];
+    const int row = re.row, draft = re.draft;
+    const int b = row / a.W;
     RowScratch* rs = a.scratch + row;
-    if (i >= L) {
-      if (tid == 0) {
-        a.out_cnt[row] = 0;
-        *rs = RowScratch{0.0f, -1, 0.0f, 0};
-      }
-      continue;
-    }
     const int kcap = a.kcap;
-    const int draft = a.drafts ? a.drafts[row] : -1;
     // the row's own random number: needed last, computed while waiting
-    const int pos = (a.pos_base ? a.pos_base[b] : 0) + i;
-    const int iter = a.iteration ? a.iteration[b] : a.iteration0;
-    const Philox4 rnd = philox4x32_10((uint32_t)pos, (uint32_t)(a.seq_base + b), (uint32_t)iter, (uint32_t)a.purpose,
+    const Philox4 rnd = philox4x32_10((uint32_t)re.pos, (uint32_t)(a.seq_base + b), (uint32_t)re.iter, (uint32_t)a.purpose,
                                       a.seed_lo, a.seed_hi);
-    if (!dead) dead = !mbar_wait(sm.cand_full, n_row & 1u);
+    if (!dead) dead = !mbar_wait_abortable(sm.cand_full, (uint32_t)k & 1u, abort_flag);
     dead = group_any<NT_P, BAR_P>(dead || (*abort_flag != 0));
     if (dead) {
       if (tid == 0) {
@@ -514,93 +745,122 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       }
       continue;
     }
+    SJD_PHASE(16);
     const float tau0 = __int_as_float(sm.ctl[kRcRowTau0]);
-    const float vmax = __int_as_float(sm.ctl[kRcRowVmax]);
-    const uint32_t n_total = (uint32_t)sm.ctl[kRcRowTotal];
+    const float top = __int_as_float(sm.ctl[kRcRowTop]);
+    const uint32_t n_pairs = (uint32_t)sm.ctl[kRcRowPairs];
     bool fallback = kcap > kKcapMax || sm.ctl[kRcRowFallback] != 0;
-    ++n_row;
     if (fallback) {
       // exact any-shape path from global memory (the row is still in L2); its scratch sits on st_vals, so
       // that the bins (= st_ids) stay clear
       group_sync<NT_P, BAR_P>();
       if (tid == 0) mbar_arrive(sm.cand_free);
-      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals), kRowStatusRedone);
+      redo_row<DTYPE, NT_P, BAR_P>(a, row, tid, sm.st_vals);
       continue;
     }
-    // linear bins over [tau0, vmax]; monotone in y, so a higher bin never holds a smaller value
-    const float range = __fsub_rn(vmax, tau0);
+    // ---- every thread takes an equal share of the pair list: a run of consecutive pairs, so that
+    // concatenating the threads' survivors keeps the id order.  Linear bins over [tau0, top] (top: the largest
+    // sample value; anything above it lands in the last bin); monotone in y, so a higher bin never holds a
+    // smaller value.  A thread keeps the bins of its values in registers: 0 = below tau0 (not a candidate),
+    // otherwise bin + 1.
+    const float range = __fsub_rn(top, tau0);
     const float scale = range > 0.0f ? __fdiv_rn((float)kSelBins * 0.999f, range) : 0.0f;
-    auto bin_of = [&](float y) {
-      const int q = __float2int_rd(__fmul_rn(__fsub_rn(y, tau0), scale));
-      return min(max(q, 0), kSelBins - 1);
-    };
+    const uint32_t chunk = (n_pairs + NT_P - 1) / NT_P;  // <= kPairChunk
+    const uint32_t my_first = min((uint32_t)tid * chunk, n_pairs);
+    const uint32_t my_count = min(my_first + chunk, n_pairs) - my_first;
     if (tid == 0) {
       sm.ctl[kRcGather] = 0;
       sm.ctl[kRcPtok] = 0;
       sm.ctl[kRcFoundId] = -1;
     }
-    // every candidate into its bin, four independent entries per thread in flight
-    for (uint32_t i0 = 0; i0 < n_total; i0 += 4 * NT_P) {
-      float yv[4];
-      bool v[4];
+    uint32_t code[kPairChunk];
+    float vmax = neg_inf;
+    constexpr int kHalf = (kPairChunk + 1) / 2;  // loads in flight together
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint32_t ix = i0 + q * NT_P + tid;
-        v[q] = ix < n_total;
-        if (v[q]) yv[q] = sm.dense[ix].y;
-      }
+    for (int j0 = 0; j0 < kPairChunk; j0 += kHalf) {
+      // loads first (a slot beyond the thread's share reads a valid address and is masked out)
+      float2 v[kHalf];
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        if (v[q]) atomicAdd(&sm.sel[bin_of(yv[q])], 1u);
-    }
-    group_sync<NT_P, BAR_P>();
-    // ---- exact K-th largest: threshold bin, then ranking inside it by (y descending, id ascending) ----
-    int tbin = 0, need = 0, nbin = 0;
-    find_rank_bin<kSelBins, NT_P, BAR_P>(sm.sel, (uint32_t)kcap, tid, sm.scan_p, flip, sm.ctl, kRcPBin);
-    if (!fallback) {
-      tbin = sm.ctl[kRcPBin];
-      need = kcap - sm.ctl[kRcPAbove];  // members of the threshold bin that survive
-      nbin = sm.ctl[kRcPCount];
-      if (tbin < 0 || nbin > kBinListCap) fallback = true;
-    }
-    // from here on every thread works on an equal share of the dense list: a run of consecutive entries,
-    // so that concatenating the threads' survivors keeps the id order
-    const uint32_t chunk = (n_total + NT_P - 1) / NT_P;
-    const uint32_t my_first = fallback ? 0u : min((uint32_t)tid * chunk, n_total);
-    const uint32_t my_count = fallback ? 0u : min(my_first + chunk, n_total) - my_first;
-    uint32_t n_above = 0, n_in_bin = 0;
-    if (!fallback) {
-      for (uint32_t k = 0; k < my_count; ++k) {
-        const Candidate c = sm.dense[my_first + k];
-        const int q = bin_of(c.y);
-        if (q > tbin) ++n_above;
-        else if (q == tbin) {
-          ++n_in_bin;
-          sm.binlist[atomicAdd(&sm.ctl[kRcGather], 1)] = BinMember{c.y, (int32_t)(my_first + k)};
+      for (int u = 0; u < kHalf; ++u)
+        if (j0 + u < kPairChunk)
+          v[u] = *reinterpret_cast<const float2*>(&sm.pair_y[min(my_first + (uint32_t)(j0 + u), (uint32_t)kRangePairCap - 1u)]);
+#pragma unroll
+      for (int u = 0; u < kHalf; ++u) {
+        if (j0 + u < kPairChunk) {
+          const bool mine = (uint32_t)(j0 + u) < my_count;
+          const bool v0 = mine && v[u].x >= tau0, v1 = mine && v[u].y >= tau0;  // false for NaN
+          const int q0 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[u].x, tau0), scale)), kSelBins - 1);
+          const int q1 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[u].y, tau0), scale)), kSelBins - 1);
+          const uint32_t c0 = v0 ? (uint32_t)q0 + 1u : 0u, c1 = v1 ? (uint32_t)q1 + 1u : 0u;
+          code[j0 + u] = c0 | (c1 << 16);
+          vmax = fmaxf(vmax, v0 ? v[u].x : neg_inf);
+          vmax = fmaxf(vmax, v1 ? v[u].y : neg_inf);
+          if (c0 != 0u) atomicAdd(&sm.sel[c0 - 1u], 1u);
+          if (c1 != 0u) atomicAdd(&sm.sel[c1 - 1u], 1u);
         }
       }
     }
+    // the row's maximum: per warp here, combined after the barriers of the search below
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, d));
+    float* const warp_max = reinterpret_cast<float*>(sm.scan_p + 64);
+    if (lane == 0) warp_max[warp - NF] = vmax;
+    group_sync<NT_P, BAR_P>();
+    SJD_PHASE(17);
+    // ---- exact K-th largest: threshold bin, then ranking inside it by (y descending, id ascending) ----
+    find_rank_bin<kSelBins, NT_P, BAR_P>(sm.sel, (uint32_t)kcap, tid, sm.scan_p, flip, sm.ctl, kRcPBin);
+    const int tbin = sm.ctl[kRcPBin];
+    const int need = kcap - sm.ctl[kRcPAbove];  // members of the threshold bin that survive
+    const int nbin = sm.ctl[kRcPCount];
+#pragma unroll
+    for (int w = 0; w < NP; ++w) vmax = fmaxf(vmax, warp_max[w]);
+    // fewer than kcap candidates (the sampled threshold was too high), a threshold bin too crowded for the
+    // on-chip ranking, or no finite maximum: the any-shape path redoes the row
+    if (tbin < 0 || nbin > kBinListCap || !(vmax <= 3.402823466e38f)) fallback = true;
+    SJD_PHASE(18);
+    uint32_t n_above = 0;
+    bool in_bin = false;
+    if (!fallback) {
+      const uint32_t tcode = (uint32_t)tbin + 1u;
+      uint32_t hits = 0;  // bit 2j + h: value h of pair j lies in the threshold bin
+#pragma unroll
+      for (int j = 0; j < kPairChunk; ++j) {
+        const uint32_t c0 = code[j] & 0xffffu, c1 = code[j] >> 16;
+        n_above += (c0 > tcode ? 1u : 0u) + (c1 > tcode ? 1u : 0u);
+        hits |= (c0 == tcode ? 1u : 0u) << (2 * j);
+        hits |= (c1 == tcode ? 1u : 0u) << (2 * j + 1);
+      }
+      in_bin = hits != 0u;
+      while (hits != 0u) {  // a handful of values per row
+        const int bit = __ffs((int)hits) - 1;
+        hits &= hits - 1u;
+        const int slot = (int)(2u * my_first) + bit;
+        sm.binlist[atomicAdd(&sm.ctl[kRcGather], 1)] = BinMember{pair_vals[slot], slot};
+      }
+    }
     group_sync<NT_P, BAR_P>();
     if (!fallback) {
-      // losers of the threshold bin are struck from the dense list: the sign bit of their id is set
+      // losers of the threshold bin are struck from the pair list: their value becomes -inf
       for (int x = tid; x < nbin; x += NT_P) {
         const BinMember me = sm.binlist[x];
-        const int my_id = sm.dense[me.slot].id & 0x7fffffff;
         int rank = 0;
         for (int z = 0; z < nbin; ++z) {
           const BinMember o = sm.binlist[z];
-          const int o_id = sm.dense[o.slot].id & 0x7fffffff;
-          rank += (o.y > me.y || (o.y == me.y && o_id < my_id)) ? 1 : 0;
+          rank += (o.y > me.y || (o.y == me.y && o.slot < me.slot)) ? 1 : 0;
         }
-        if (rank >= need) sm.dense[me.slot].id = my_id | (int)0x80000000;
+        if (rank >= need) pair_vals[me.slot] = neg_inf;
       }
     }
     group_sync<NT_P, BAR_P>();
+    SJD_PHASE(19);
     uint32_t my_alive = n_above;
-    if (n_in_bin != 0u) {
-      for (uint32_t k = 0; k < my_count; ++k) {
-        const Candidate c = sm.dense[my_first + k];
-        if (c.id >= 0 && bin_of(c.y) == tbin) ++my_alive;
+    if (in_bin) {
+      const uint32_t tcode = (uint32_t)tbin + 1u;
+#pragma unroll
+      for (int j = 0; j < kPairChunk; ++j) {
+        const uint32_t c0 = code[j] & 0xffffu, c1 = code[j] >> 16;
+        if (c0 == tcode && pair_vals[2u * (my_first + j)] >= tau0) ++my_alive;
+        if (c1 == tcode && pair_vals[2u * (my_first + j) + 1u] >= tau0) ++my_alive;
       }
     }
     uint32_t total_alive;
@@ -608,23 +868,46 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     if (!fallback && total_alive != (uint32_t)kcap) fallback = true;  // cannot happen; keep the result exact anyway
     if (!fallback) {
       // ---- survivors, already in ascending id order (this overwrites sel and binlist) ----
-      for (uint32_t k = 0; k < my_count; ++k) {
-        const Candidate c = sm.dense[my_first + k];
-        if (c.id >= 0 && bin_of(c.y) >= tbin) {
-          sm.st_ids[out_pos] = c.id;
-          sm.st_vals[out_pos] = c.y;
-          ++out_pos;
+      const uint32_t tcode = (uint32_t)tbin + 1u;
+#pragma unroll
+      for (int j0 = 0; j0 < kPairChunk; j0 += kHalf) {
+        float2 v[kHalf];
+        int id[kHalf];
+#pragma unroll
+        for (int u = 0; u < kHalf; ++u) {
+          if (j0 + u < kPairChunk) {
+            const uint32_t at = min(my_first + (uint32_t)(j0 + u), (uint32_t)kRangePairCap - 1u);
+            v[u] = *reinterpret_cast<const float2*>(&sm.pair_y[at]);
+            id[u] = 2 * (int)sm.pair_q[at];
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kHalf; ++u) {
+          if (j0 + u < kPairChunk) {
+            const uint32_t c0 = code[j0 + u] & 0xffffu, c1 = code[j0 + u] >> 16;
+            if (c0 > tcode || (c0 == tcode && v[u].x >= tau0)) {
+              sm.st_ids[out_pos] = id[u];
+              sm.st_vals[out_pos] = canonical(v[u].x);
+              ++out_pos;
+            }
+            if (c1 > tcode || (c1 == tcode && v[u].y >= tau0)) {
+              sm.st_ids[out_pos] = id[u] + 1;
+              sm.st_vals[out_pos] = canonical(v[u].y);
+              ++out_pos;
+            }
+          }
         }
       }
     }
     group_sync<NT_P, BAR_P>();
-    // the dense list is not read again: hand it back
+    SJD_PHASE(20);
+    // the pair list is not read again: hand it back
     if (tid == 0) mbar_arrive(sm.cand_free);
     if (fallback) {
-      // the threshold bin was too crowded for the on-chip ranking: exact any-shape path from global memory.
-      // The bins were cleared when they were read; the any-shape path's scratch sits on st_vals.
+      // exact any-shape path from global memory.  The bins were cleared when they were read; the any-shape
+      // path's scratch sits on st_vals.
       for (int j = tid; j < kSelBins; j += NT_P) sm.sel[j] = 0;
-      row_generic<DTYPE, NT_P, BAR_P>(a, row, tid, *reinterpret_cast<GenericSmem*>(sm.st_vals), kRowStatusRedone);
+      redo_row<DTYPE, NT_P, BAR_P>(a, row, tid, sm.st_vals);
       continue;
     }
     // ---- normalise, write the row, draw from it ----
@@ -643,13 +926,15 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     *reinterpret_cast<uint4*>(sm.sel + k0) = make_uint4(0u, 0u, 0u, 0u);
     *reinterpret_cast<uint4*>(sm.sel + k0 + 4) = make_uint4(0u, 0u, 0u, 0u);
     const float Z = group_sum1_f32<NT_P, BAR_P>(zpart, tid, sm.scan_p, flip);
+    SJD_PHASE(21);
     int32_t* out_ids = a.out_ids + (size_t)row * kcap;
     float* out_vals = a.out_vals + (size_t)row * kcap;
     uint64_t wgt[kFinItems], wloc = 0;
     float p[kFinItems];
+    const float inv_Z = __fdiv_rn(1.0f, Z);  // one division per thread; p = e / Z within 1.5 ulp
 #pragma unroll
     for (int j = 0; j < kFinItems; ++j) {
-      p[j] = __fdiv_rn(e[j], Z);
+      p[j] = __fmul_rn(e[j], inv_Z);
       wgt[j] = fixed_weight(p[j]);
       wloc += wgt[j];
       if (ids[j] == draft && ids[j] >= 0) sm.ctl[kRcPtok] = __float_as_int(p[j]);
@@ -670,6 +955,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
         }
       }
     }
+    SJD_PHASE(22);
     // the row's own draw from p_i: fixed-point inverse CDF in ascending-id order
     uint64_t T;
     const uint64_t lo = group_scan1<NT_P, BAR_P, uint64_t>(wloc, tid, sm.scan_p, flip, &T);
@@ -705,6 +991,9 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       *rs = RowScratch{__int_as_float(sm.ctl[kRcPtok]), sm.ctl[kRcFoundId], __int_as_float(sm.ctl[kRcFoundP]), 0};
     }
     group_sync<NT_P, BAR_P>();
+    SJD_PHASE(23);
+    SJD_PHASE_COUNT(40, 1);
+    SJD_PHASE_COUNT(41, n_pairs);
   }
 }
 

@@ -9,6 +9,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "device_once.h"
 #include "device_utils.cuh"
 #include "row_kernels.cuh"
 #include "rows_pipeline.cuh"
@@ -31,17 +32,32 @@ int cuda_fail(cudaError_t e, const char* what) {
 constexpr int kGenericThreads = 512;
 constexpr int kVerifyThreads = 512;
 
+int current_device() {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
+// SM count of the current device (cached per device ordinal).
 int sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      cached = n;
-    else
-      return 148;
-  }
-  return cached;
+  static sjd::DeviceValue cache;
+  const int dev = current_device();
+  const int n = cache.get(dev, [dev] {
+    int v = 0;
+    return (dev >= 0 && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) ? v : 0;
+  });
+  return n > 0 ? n : 148;
+}
+
+// The opt-in to more than 48 KB of dynamic shared memory belongs to the (device, kernel) pair: it is set
+// once per device for each kernel instantiation (`once` is that instantiation's record).
+template <typename Kern>
+cudaError_t allow_large_smem(Kern kern, sjd::DeviceOnce& once, int bytes) {
+  cudaError_t err = cudaSuccess;
+  once.run_once(current_device(), [&] {
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return err == cudaSuccess ? 0 : 1;
+  });
+  return err;
 }
 
 constexpr int kFilterWarps = 8;
@@ -147,18 +163,27 @@ bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem
   const int m = sample_rank(a);
   if (m > n_sample / 2) return false;
   const int sample_all = m > n_sample / 8 ? 1 : 0;  // the rank must exist among what the first pass bins
-  const double mean = (double)m * S, sd = (double)S * std::sqrt((double)m);
-  if (mean + 4.0 * sd > (double)sjd::kRangeDenseCap) return false;
-  // pair entries: the candidates outside the sample, and the sample kept against a floor below its rank-m
-  // element (the floor from group maxima lies lower than the one from every element)
-  const double per_thread = (mean * (S - 1) / S + (sample_all ? 1.7 : 2.1) * m) / sjd::kRangeThreads;
-  if (per_thread + 5.0 * std::sqrt(per_thread) + 1.0 > (double)(sjd::kListCap - 4)) return false;
+  // candidates of a row: m S on average; pairs of neighbours with at least one candidate: a little fewer
+  const double cand = (double)m * S, cand_sd = (double)S * std::sqrt((double)m);
+  const double thin = 1.0 - 0.5 * cand / V;
+  if ((cand + 5.0 * cand_sd) * thin > (double)sjd::kRangePairCap) return false;
+  // pair entries per filter thread: a Poisson count; its list must hold it with a tail below 1e-6
+  const double per_thread = cand * thin / sjd::kRangeThreads;
+  if (per_thread + 5.0 * std::sqrt(per_thread) + 1.0 > (double)(sjd::kRangeListCap - 4)) return false;
   if (need_encoder && encode_tiled_fn() == nullptr) return false;
   cfg->sample_rank = m;
   cfg->sample_all = sample_all;
+  // the element rank m as a rank among the maxima of the sample's groups of eight (see the sampler); only
+  // while at most a tenth of the sample lies above the threshold, beyond that the group maxima resolve it badly
+  {
+    const double p = (double)m / n_sample, groups = n_sample / 8.0;
+    cfg->group_rank = (!sample_all && p <= 0.10) ? (int)std::ceil(groups * (1.0 - std::pow(1.0 - p, 8.0))) : 0;
+  }
   cfg->stages = S;
   cfg->range_len = R;
   cfg->mask_words = mask_words;
+  cfg->row_begin = 0;
+  cfg->row_end = P->B * P->W;
   *smem = sjd::range_smem_bytes(mask_words);
   return *smem <= kSmemLimit;
 }
@@ -199,28 +224,25 @@ cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&lc, kern, std::forward<Args>(args)...);
 }
 
+constexpr int kSamplerWarps = 4;
+
 template <int DTYPE>
 cudaError_t launch_ranges(const sjd::RowArgs& ra, const sjd::RangeCfg& cfg, const CUtensorMap& mc, const CUtensorMap& mu,
                           size_t smem, int grid, cudaStream_t st) {
-  auto kern = sjd::rows_ranges_kernel<DTYPE, kFinisherWarps>;
-  static bool configured = false;  // per instantiation; the attribute is sticky for the process
-  if (!configured) {
-    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  return launch_after(kern, dim3((unsigned)grid), dim3((8 + kFinisherWarps + 1) * 32), smem, st, true, ra, cfg, mc, mu);
+  auto kern = sjd::rows_ranges_kernel<DTYPE, kFinisherWarps, kSamplerWarps>;
+  static sjd::DeviceOnce configured;  // per instantiation
+  const cudaError_t e = allow_large_smem(kern, configured, (int)kSmemLimit);
+  if (e != cudaSuccess) return e;
+  return launch_after(kern, dim3((unsigned)grid), dim3((8 + kFinisherWarps + kSamplerWarps + 1) * 32), smem, st, true, ra,
+                      cfg, mc, mu);
 }
 
 template <int DTYPE>
 cudaError_t launch_pipeline(const sjd::RowArgs& ra, const sjd::PipeCfg& cfg, size_t smem, int grid, cudaStream_t st) {
   auto kern = sjd::rows_pipeline_kernel<DTYPE, kFilterWarps, kFinisherWarps>;
-  static bool configured = false;  // per instantiation; the attribute is sticky for the process
-  if (!configured) {
-    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static sjd::DeviceOnce configured;  // per instantiation
+  const cudaError_t e = allow_large_smem(kern, configured, (int)kSmemLimit);
+  if (e != cudaSuccess) return e;
   return launch_after(kern, dim3((unsigned)grid), dim3((kFilterWarps + kFinisherWarps + 1) * 32), smem, st, true, ra, cfg);
 }
 
@@ -229,7 +251,7 @@ cudaError_t launch_pipeline(const sjd::RowArgs& ra, const sjd::PipeCfg& cfg, siz
 constexpr size_t kStaticScratchBytes = (((size_t)SJD_STATIC_MAX_ROWS * sizeof(sjd::RowScratch) + 256) + 255) & ~(size_t)255;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
+using sjd::kMaxDevices;
 std::mutex g_static_mutex;
 void* g_static_scratch_addr[kMaxDevices] = {};  // device address of g_static_scratch, per device ordinal
 
@@ -283,6 +305,20 @@ const char* sjd_status_string(int code) {
 const char* sjd_last_cuda_error(void) { return g_cuda_error; }
 
 uint64_t sjd_launch_count(void) { return g_launches.load(); }
+
+#ifdef SJD_PHASE_TIMERS
+// Diagnostic builds only: copies the 48 phase counters to `out` (host) after a device synchronisation and
+// optionally clears them.
+int sjd_phase_cycles_read(unsigned long long* out, int reset) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return SJD_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(out, sjd::g_phase_cycles, sizeof(unsigned long long) * 48) != cudaSuccess) return SJD_ERR_CUDA;
+  if (reset) {
+    unsigned long long z[48] = {0};
+    if (cudaMemcpyToSymbol(sjd::g_phase_cycles, z, sizeof(z)) != cudaSuccess) return SJD_ERR_CUDA;
+  }
+  return SJD_OK;
+}
+#endif
 
 size_t sjd_workspace_bytes(const sjd_params* p) {
   if (!p || p->B < 0 || p->W < 1) return 0;
@@ -350,10 +386,19 @@ int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* 
     const bool fast = !(P->flags & (SJD_FLAG_FORCE_GENERIC | SJD_FLAG_FORCE_TILES));
     if (fast && plan_ranges(P, kcap, &rcfg, &smem) && make_range_map(&map_c, logits_cond, P, rcfg) &&
         make_range_map(&map_u, logits_uncond ? logits_uncond : logits_cond, P, rcfg)) {
-      const int grid = rows < sm_count() ? rows : sm_count();
-      e = P->logits_dtype == SJD_BF16  ? launch_ranges<1>(ra, rcfg, map_c, map_u, smem, grid, stream)
-          : P->logits_dtype == SJD_F16 ? launch_ranges<2>(ra, rcfg, map_c, map_u, smem, grid, stream)
-                                       : launch_ranges<0>(ra, rcfg, map_c, map_u, smem, grid, stream);
+      // a CTA takes at most kRowsPerCta rows per launch: larger problems go in several launches
+      const int per_launch = sjd::kRowsPerCta * sm_count();
+      e = cudaSuccess;
+      for (int r0 = 0; r0 < rows && e == cudaSuccess; r0 += per_launch) {
+        rcfg.row_begin = r0;
+        rcfg.row_end = r0 + per_launch < rows ? r0 + per_launch : rows;
+        const int n = rcfg.row_end - r0;
+        const int grid = n < sm_count() ? n : sm_count();
+        e = P->logits_dtype == SJD_BF16  ? launch_ranges<1>(ra, rcfg, map_c, map_u, smem, grid, stream)
+            : P->logits_dtype == SJD_F16 ? launch_ranges<2>(ra, rcfg, map_c, map_u, smem, grid, stream)
+                                         : launch_ranges<0>(ra, rcfg, map_c, map_u, smem, grid, stream);
+        if (e == cudaSuccess && r0 > 0) ++g_launches;
+      }
     } else if (!(P->flags & SJD_FLAG_FORCE_GENERIC) && plan_pipeline(P, kcap, &cfg, &smem)) {
       const int grid = rows < sm_count() ? rows : sm_count();
       e = P->logits_dtype == SJD_BF16  ? launch_pipeline<1>(ra, cfg, smem, grid, stream)
