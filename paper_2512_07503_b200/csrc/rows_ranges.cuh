@@ -63,7 +63,6 @@ constexpr int kRangeRingStages = 3;
 constexpr int kRangeListCap = 35;           // pair entries per filter thread and row (the last four are slack for
                                             // the unconditional stores of one group)
 constexpr int kRangePairCap = 3328;         // candidate pairs the finisher can hold for a row
-constexpr int kPairChunk = (kRangePairCap + kRangeThreads - 1) / kRangeThreads;  // pairs per finisher thread
 constexpr int kSampleBins = 1024;           // sampler's histogram (group maxima by key, then linear bins)
 constexpr int kSampleKeyShift = 22;         // key bits dropped by the first histogram: sign, exponent, one mantissa bit
 constexpr int kRowsPerCta = 32;             // live rows a CTA takes in one launch (the host splits larger problems)
@@ -86,7 +85,7 @@ enum {
   kRcTau0, kRcTau1, kRcTau2, kRcTau3,                   // tau0 of live row k in word kRcTau0 + (k & 3)
   kRcTop0, kRcTop1, kRcTop2, kRcTop3,                   // largest sample value of live row k, likewise
   kRcRowTau0, kRcRowTop, kRcRowPairs, kRcRowFallback,   // handed over with the row
-  kRcPBin, kRcPAbove, kRcPCount, kRcGather, kRcPtok, kRcFoundId, kRcFoundP,  // finisher
+  kRcPBin, kRcPAbove, kRcPCount, kRcGather, kRcPtok, kRcFoundId, kRcFoundP, kRcRedo,  // finisher
   kRcWords = 32
 };
 
@@ -114,6 +113,7 @@ struct RangeSmem {
   BinMember* binlist;   // [kBinListCap] = st_vals: likewise
   uint32_t* hist;       // [kSampleBins] sampler
   RowEntry* tab;        // [kRowsPerCta]
+  int32_t* redo;        // [kRowsPerCta] rows the single pass could not finish (redone at the end)
   uint64_t* full;       // [kRangeRingStages] a row stage has landed in the slot (waited for by the filter)
   uint64_t* empty;      // [kRangeRingStages] the slot's eight consumer warps are done with it
   uint64_t* sample_full;  // [2] a sample has landed in its slot (row parity; waited for by the sampler)
@@ -135,6 +135,7 @@ __host__ __device__ inline size_t range_smem_bytes(int mask_words) {
   b += (size_t)kKcapMax * 8;
   b += (size_t)kSampleBins * 4;
   b += (size_t)kRowsPerCta * sizeof(RowEntry);
+  b += (size_t)kRowsPerCta * 4;
   b += 16 * 8 + 3 * (2 * 32 + 8) * 8 + kRcWords * 4;
   return b;
 }
@@ -165,6 +166,8 @@ __device__ __forceinline__ RangeSmem carve_range_smem(unsigned char* base, int m
   p += (size_t)mask_words * kRangeThreads * 4;
   s.tab = reinterpret_cast<RowEntry*>(p);
   p += (size_t)kRowsPerCta * sizeof(RowEntry);
+  s.redo = reinterpret_cast<int32_t*>(p);
+  p += (size_t)kRowsPerCta * 4;
   s.full = reinterpret_cast<uint64_t*>(p);
   s.empty = s.full + kRangeRingStages;
   s.sample_full = s.empty + kRangeRingStages;
@@ -242,6 +245,85 @@ __device__ __forceinline__ void tma_load_box(void* dst, const CUtensorMap* map, 
       : "memory");
 }
 
+// Largest bin b with (entries in bins > b) < target <= (entries in bins >= b), found by ONE warp without a
+// barrier: lane l sums bins [P (31 - l), P (32 - l)) with P = BINS / 32, a scan over the lanes finds the lane
+// whose bins hold the rank, and that lane's P bins are spread over the lanes for a second scan.  Every lane
+// gets the result: bin + 1 in bits 0-11 of one word (0 when the histogram holds fewer than `target`
+// entries) with the bin's own count in bits 12-31, and the count above the bin.  Counts stay below 2^20 (a
+// row has at most 2^17 values).  With ZERO the warp also clears the histogram (it must be the only reader).
+// Inlined on purpose, like everything on the roles' paths: an out-of-line function saves and restores
+// registers through local memory, and local memory lies behind the ring's outstanding copies.
+struct RankBin {
+  uint32_t bin_count;  // (count << 12) | (bin + 1)
+  uint32_t above;
+  __device__ __forceinline__ int bin() const { return (int)(bin_count & 0xfffu) - 1; }
+  __device__ __forceinline__ uint32_t count() const { return bin_count >> 12; }
+};
+template <int BINS, bool ZERO>
+__device__ __forceinline__ uint2 warp_rank_bin_raw(uint32_t* hist, uint32_t target, int lane) {
+  constexpr int P = BINS / 32;   // bins per lane
+  constexpr int Q = P / 32;      // bins per lane of the second step
+  static_assert(BINS % 1024 == 0 && (Q == 1 || Q == 2), "1024 or 2048 bins");
+  // a lane's bins lie P words apart from its neighbour's, i.e. in the same banks: every lane starts its walk
+  // at a different 16-byte piece, so that the eight lanes served together touch eight different bank groups
+  uint4* mine = reinterpret_cast<uint4*>(hist + P * (31 - lane));
+  uint32_t sum = 0;
+#pragma unroll
+  for (int x = 0; x < P / 4; ++x) {
+    const uint4 w = mine[(x + lane) & (P / 4 - 1)];
+    sum += w.x + w.y + w.z + w.w;
+  }
+  uint32_t inc = sum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t n = __shfl_up_sync(0xffffffffu, inc, d);
+    if (lane >= d) inc += n;
+  }
+  const uint32_t owner_votes = __ballot_sync(0xffffffffu, inc - sum < target && target <= inc);
+  uint2 result = make_uint2(0u, 0u);
+  if (owner_votes != 0u) {
+    const int owner = __ffs((int)owner_votes) - 1;
+    const uint32_t above0 = __shfl_sync(0xffffffffu, inc - sum, owner);  // entries in bins above the owner's
+    const int seg = P * (31 - owner);                                     // the owner's bins: [seg, seg + P)
+    // lane l takes the Q bins ending at seg + P - 1 - Q l (descending with l); c_hi is the upper one
+    uint32_t c_lo, c_hi;
+    if (Q == 2) {
+      const uint2 c = *reinterpret_cast<const uint2*>(hist + seg + P - 2 - 2 * lane);
+      c_lo = c.x;
+      c_hi = c.y;
+    } else {
+      c_hi = hist[seg + P - 1 - lane];
+      c_lo = 0;
+    }
+    const uint32_t both = c_lo + c_hi;
+    uint32_t inc2 = both;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, inc2, d);
+      if (lane >= d) inc2 += n;
+    }
+    const uint32_t ab = above0 + inc2 - both;  // above this lane's upper bin
+    const bool in_hi = ab < target && target <= ab + c_hi;
+    const bool in_lo = Q == 2 && ab + c_hi < target && target <= ab + both;
+    const int l2 = __ffs((int)__ballot_sync(0xffffffffu, in_hi || in_lo)) - 1;  // exists: the owner's bins hold the rank
+    const uint32_t my_bin = (uint32_t)(seg + P - Q - Q * lane + ((Q == 2 && in_hi) ? 1 : 0));
+    const uint32_t my_cnt = in_hi ? c_hi : c_lo;
+    result.x = __shfl_sync(0xffffffffu, (my_cnt << 12) | (my_bin + 1u), l2);
+    result.y = __shfl_sync(0xffffffffu, in_hi ? ab : ab + c_hi, l2);
+  }
+  if (ZERO) {
+    __syncwarp();
+#pragma unroll
+    for (int x = 0; x < P / 4; ++x) mine[(x + lane) & (P / 4 - 1)] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  return result;
+}
+template <int BINS, bool ZERO>
+__device__ __forceinline__ RankBin warp_rank_bin(uint32_t* hist, uint32_t target, int lane) {
+  const uint2 r = warp_rank_bin_raw<BINS, ZERO>(hist, target, lane);
+  return RankBin{r.x, r.y};
+}
+
 // ---------------------------------------------------------------------------------------------------
 // what the three consumer roles share: how a thread finds its 64 bytes of a staged slice
 // ---------------------------------------------------------------------------------------------------
@@ -281,24 +363,23 @@ struct StageReader {
 // Either way the ring slot is given back as soon as the sample is in registers.  tau0 only steers how many
 // candidates the filter keeps (the result is exact whatever it is; too few candidates send the row to the
 // any-shape path), so neither the rounding to 11 bits nor the translation of the rank costs exactness.
-// Sampler thread t looks after ranges t and t + 128.
+// Sampler thread t looks after ranges t, t + NT, t + 2 NT, ... (NT sampler threads; the last round may be short).
 template <int DTYPE, bool HAS_U, bool HAS_T, bool BY_GROUPS, int NA>
 __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const RangeCfg& cfg, const RangeSmem& sm, int tid) {
   constexpr int NT_A = NA * 32;
   constexpr int BAR_A = 3;
-  constexpr int TI = DTYPE != 0 ? 4 : 2;        // groups of eight elements per range in stage 0
-  constexpr int NR = kRangeThreads / NT_A;       // ranges per sampler thread
-  constexpr int NG = NR * TI;                    // groups per sampler thread
-  static_assert(kRangeThreads % NT_A == 0, "ranges must split evenly over the sampler threads");
-  const int lane = tid & 31;
+  constexpr int TI = DTYPE != 0 ? 4 : 2;                     // groups of eight elements per range in stage 0
+  constexpr int NR = (kRangeThreads + NT_A - 1) / NT_A;       // ranges per sampler thread (at most)
+  constexpr int NG = NR * TI;                                 // groups per sampler thread (at most)
+  const int lane = tid & 31, warp_a = tid >> 5;
   const float neg_inf = __int_as_float(0xff800000);
   const float lowest = -3.402823466e38f;  // with this threshold every finite value is a candidate
   volatile int* abort_flag = sm.ctl + kRcAbort;
   const uint64_t s2 = pack2(a.s, a.s), t2 = pack2(a.inv_T, a.inv_T);
   const uint32_t ring_addr = smem_u32(sm.ring);
   const uint32_t n_live = (uint32_t)sm.ctl[kRcLive];
+  const uint32_t rank = (uint32_t)(BY_GROUPS ? cfg.group_rank : cfg.sample_rank);
   RingPos pos{0, 0};
-  int flip = 0;
   for (uint32_t k = 0; k < n_live; ++k) {  // live rows of this CTA
     SJD_PHASE_BEGIN();
     // ---------------- the sample into registers; first pass on the way: maxima of groups of eight, by key ----------------
@@ -307,44 +388,59 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
     __half2 cache[BY_GROUPS ? 1 : NG * 4];
     float gmax[NG];
     float smax = neg_inf;
-    constexpr bool by_groups = BY_GROUPS;
-    const uint32_t rank = (uint32_t)(by_groups ? cfg.group_rank : cfg.sample_rank);
 #pragma unroll
     for (int g = 0; g < NG; ++g) gmax[g] = neg_inf;
     if (ok) {
       const uint32_t stage0 = ring_addr + (uint32_t)pos.slot * (2 * kRangeStageBytes);
+      // one group of eight per round.  The loop is kept rolled (the code of all roles has to stay in the
+      // instruction cache): what a round finds is pushed in at the front of gmax / cache, the older entries move up.
+#pragma unroll 1
+      for (int g = 0; g < NG; ++g) {
+        const int r = g / TI, j = g % TI;
+        // a thread without a range in the last round works on a copy of range 255 and counts nothing (the
+        // warp stays together for the vote below)
+        const bool have = tid + r * NT_A < kRangeThreads;
+        const StageReader<DTYPE, HAS_U> rd(have ? tid + r * NT_A : kRangeThreads - 1);
 #pragma unroll
-      for (int r = 0; r < NR; ++r) {
-        const StageReader<DTYPE, HAS_U> rd(tid + r * NT_A);
+        for (int x = NG - 1; x >= 1; --x) gmax[x] = gmax[x - 1];
+        if (!BY_GROUPS) {
 #pragma unroll
-        for (int j = 0; j < TI; ++j) {
-          RawTile<DTYPE> raw;
-          rd.load_group(stage0, j, raw);
-          float y[8];
-          merge_raw<DTYPE, HAS_U, HAS_T>(raw, s2, t2, y);
-          const float m8 = canonical(max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]));
-          gmax[r * TI + j] = m8;
-          if (!by_groups) {
+          for (int x = NG * 4 - 1; x >= 4; --x) cache[BY_GROUPS ? 0 : x] = cache[BY_GROUPS ? 0 : x - 4];
+        }
+        RawTile<DTYPE> raw;
+        rd.load_group(stage0, j, raw);
+        float y[8];
+        merge_raw<DTYPE, HAS_U, HAS_T>(raw, s2, t2, y);
+        float m8 = canonical(max3(max3(max3(neg_inf, y[0], y[1]), y[2], y[3]), max3(y[4], y[5], y[6]), y[7]));
+        if (!have) m8 = neg_inf;
+        gmax[0] = m8;
+        if (!BY_GROUPS) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) y[q] = canonical(y[q]);
+          for (int q = 0; q < 8; ++q) y[q] = have ? canonical(y[q]) : neg_inf;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) cache[BY_GROUPS ? 0 : (r * TI + j) * 4 + q] = __floats2half2_rn(y[2 * q], y[2 * q + 1]);
-          }
-          if (!BY_GROUPS && cfg.sample_all) {
+          for (int q = 0; q < 4; ++q) cache[BY_GROUPS ? 0 : q] = __floats2half2_rn(y[2 * q], y[2 * q + 1]);
+        }
+        if (!BY_GROUPS && cfg.sample_all) {
+          if (have) {
 #pragma unroll
             for (int q = 0; q < 8; ++q) atomicAdd(&sm.hist[float_key(y[q]) >> kSampleKeyShift], 1u);
-          } else {
-            // group maxima crowd into a few coarse bins: one atomic per distinct bin of the warp
-            const uint32_t bin = float_key(m8) >> kSampleKeyShift;
-            const uint32_t peers = __match_any_sync(0xffffffffu, bin);
-            if ((peers & ((1u << lane) - 1u)) == 0u) atomicAdd(&sm.hist[bin], (uint32_t)__popc(peers));
           }
-          smax = fmaxf(smax, m8);
+        } else {
+          // group maxima crowd into a few coarse bins: one atomic per distinct bin of the warp (a thread
+          // without a range votes for a bin of its own kind and adds nothing)
+          const uint32_t bin = have ? float_key(m8) >> kSampleKeyShift : 0xffffffffu;
+          const uint32_t peers = __match_any_sync(0xffffffffu, bin);
+          if (have && (peers & ((1u << lane) - 1u)) == 0u) atomicAdd(&sm.hist[bin], (uint32_t)__popc(peers));
         }
+        smax = fmaxf(smax, m8);
       }
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.empty[pos.slot], 8 / NA);  // the slot's barrier counts eight warps
+    if (lane == 0) {
+      // the slot's barrier counts eight warps: the sampler's share them out
+      const int share = 8 / NA + (warp_a < 8 % NA ? 1 : 0);
+      mbar_arrive(&sm.empty[pos.slot], (uint32_t)share);
+    }
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, d));
     if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(&sm.ctl[kRcSmaxKey]), float_key(smax));
@@ -353,9 +449,13 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
       return;
     }
     SJD_PHASE(1);
-    // at least m group maxima (or, binning everything, m elements), hence at least m sample elements, are >=
-    // the lower edge of this bin
-    find_rank_bin<kSampleBins, NT_A, BAR_A>(sm.hist, rank, tid, sm.scan_a, flip, sm.ctl, kRcABin);
+    // at least `rank` group maxima (or, binning everything, elements) are >= the lower edge of this bin.  One
+    // warp searches and clears the histogram; the others wait.
+    if (warp_a == 0) {
+      const RankBin rb = warp_rank_bin<kSampleBins, true>(sm.hist, rank, lane);
+      if (lane == 0) sm.ctl[kRcABin] = rb.bin();
+    }
+    group_sync<NT_A, BAR_A>();
     SJD_PHASE(2);
     const int cbin = sm.ctl[kRcABin];
     float floor_y = cbin >= 0 ? key_float((uint32_t)cbin << kSampleKeyShift) : lowest;
@@ -367,7 +467,7 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
     // ---------------- second pass: linear bins over [floor, sample max] ----------------
     float tau0 = lowest;
     if (refine) {
-      if (by_groups) {
+      if (BY_GROUPS) {
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
           const int bin = min(max(__float2int_rd(__fmul_rn(__fsub_rn(gmax[g], floor_y), scale)), 0), kSampleBins - 1);
@@ -385,28 +485,28 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
       }
       group_sync<NT_A, BAR_A>();
       SJD_PHASE(3);
-      if (tid == 0) sm.ctl[kRcSmaxKey] = 0;  // every thread has read it; next written after the next row's barriers
-      find_rank_bin<kSampleBins, NT_A, BAR_A>(sm.hist, rank, tid, sm.scan_a, flip, sm.ctl, kRcABin);
-      const int fbin = sm.ctl[kRcABin];
-      if (fbin > 0 && scale > 0.0f) {
-        // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
-        const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
-        tau0 = __fadd_rd(floor_y, t);
-      } else if (fbin >= 0) {
-        tau0 = floor_y;
+      if (warp_a == 0) {
+        const int fbin = warp_rank_bin<kSampleBins, true>(sm.hist, rank, lane).bin();
+        if (fbin > 0 && scale > 0.0f) {
+          // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
+          const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
+          tau0 = __fadd_rd(floor_y, t);
+        } else if (fbin >= 0) {
+          tau0 = floor_y;
+        }
       }
     } else {
-      group_sync<NT_A, BAR_A>();
-      if (tid == 0) sm.ctl[kRcSmaxKey] = 0;
+      group_sync<NT_A, BAR_A>();  // every thread has read kRcSmaxKey before it is reset below
     }
     // a word of its own for each of four consecutive rows: the filter reads it at the start of the row, and
     // the ring keeps the sampler less than two rows ahead of the filter
     if (tid == 0) {
+      sm.ctl[kRcSmaxKey] = 0;  // every thread has read it (barrier above)
       sm.ctl[kRcTau0 + (int)(k & 3u)] = __float_as_int(tau0);
       sm.ctl[kRcTop0 + (int)(k & 3u)] = __float_as_int(top_y);
       mbar_arrive(&sm.tau_full[k & 1u]);
     }
-    group_sync<NT_A, BAR_A>();  // kRcABin is rewritten by the next row's first search
+    group_sync<NT_A, BAR_A>();  // the histogram is clear and kRcSmaxKey reset before the next row's first pass
     SJD_PHASE(4);
     // sample(1) follows sample(0) directly; sample(k+1) follows sample(k) after the S stages of row k-1 and itself
     if (k == 0) pos.step();
@@ -530,7 +630,8 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
     const bool fallback = ((sum >> 14) & 0x1ffu) != 0u || n_pairs > (uint32_t)kRangePairCap;
     SJD_PHASE(11);
     if (!fallback) {
-      const uint32_t q0 = (uint32_t)(tid * (cfg.range_len >> 1));  // first pair number of this thread's range
+      uint32_t qn = (uint32_t)(tid * (cfg.range_len >> 1));  // pair number of the first bit of the current mask word
+      uint32_t y_at = smem_u32(sm.pair_y) + my_off * 8u, q_at = smem_u32(sm.pair_q) + my_off * 2u;
       int w = 0;
       uint32_t x = ~sm.masks[tid];
       for (int e0 = 0; e0 < n_e; e0 += 4) {
@@ -543,33 +644,29 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
           if (e0 + u < n_e) {
             while (x == 0u && w + 1 < mask_words) {
               ++w;
+              qn += 32u;
               x = ~sm.masks[(size_t)w * NT_F + tid];
             }
-            const int bitpos = __clz((int)x);
+            const uint32_t bitpos = (uint32_t)__clz((int)x);
             x &= ~(0x80000000u >> bitpos);
-            sm.pair_y[my_off + e0 + u] = v[u];
-            sm.pair_q[my_off + e0 + u] = (uint16_t)(q0 + (uint32_t)(w * 32 + bitpos));
+            asm volatile("st.shared.b64 [%0], %1;" ::"r"(y_at), "l"(v[u]) : "memory");
+            asm volatile("st.shared.u16 [%0], %1;" ::"r"(q_at), "h"((uint16_t)(qn + bitpos)) : "memory");
+            y_at += 8u;
+            q_at += 2u;
           }
         }
       }
     }
-    group_sync<NT_F, BAR_F>();
     if (tid == 0) {
       sm.ctl[kRcRowTau0] = __float_as_int(tau0);
       sm.ctl[kRcRowTop] = top_bits;
       sm.ctl[kRcRowPairs] = (int)n_pairs;
       sm.ctl[kRcRowFallback] = fallback ? 1 : 0;
-      mbar_arrive(sm.cand_full);
     }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(sm.cand_full);
     SJD_PHASE(12);
   }
-}
-
-// The any-shape path for a row the single pass could not finish: rare, so kept out of line (the finisher's
-// code stays small).  Its scratch sits on st_vals, so that the bins (= st_ids) stay clear.
-template <int DTYPE, int NT, int BAR>
-__device__ __noinline__ void redo_row(const RowArgs& a, int row, int tid, float* st_vals) {
-  row_generic<DTYPE, NT, BAR>(a, row, tid, *reinterpret_cast<GenericSmem*>(st_vals), kRowStatusRedone);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -582,10 +679,12 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   constexpr int NF = 8;
   constexpr int NT_F = kRangeThreads, NT_P = NP * 32;
   constexpr int BAR_P = 2;  // named barrier of the finisher warps (the filter warps use 1, the sampler warps 3)
-  constexpr int kFinItems = kKcapMax / NT_P;
+  constexpr int kFinItems = kKcapMax / NT_P;                        // staged survivors per finisher thread
+  constexpr int kPairChunk = (kRangePairCap + NT_P - 1) / NT_P;     // candidate pairs per finisher thread
   constexpr int NS = kRangeRingStages;
   constexpr int BW = 64 / (DTYPE != 0 ? 2 : 4);  // elements per stage and range
-  static_assert(NT_F == NF * 32 && NT_P == kRangeThreads && kFinItems == 8, "group sizes");
+  static_assert(NT_F == NF * 32 && kFinItems * NT_P == kKcapMax && (kFinItems == 4 || kFinItems == 8), "group sizes");
+  static_assert(2 * kPairChunk <= 32 && NP <= 16, "hit bits in one word; warp maxima in the spare scratch slots");
   extern __shared__ unsigned char smem_raw[];
   RangeSmem sm = carve_range_smem(smem_raw, cfg.mask_words);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -601,8 +700,8 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       mbar_init(&sm.sample_full[p], 1);
       mbar_init(&sm.tau_full[p], 1);
     }
-    mbar_init(sm.cand_full, 1);
-    mbar_init(sm.cand_free, 1);
+    mbar_init(sm.cand_full, NF);  // every filter warp arrives when its share of the pair list is written
+    mbar_init(sm.cand_free, NP);  // every finisher warp arrives when its share is in registers
     for (int k = 0; k < kRcWords; ++k) sm.ctl[k] = 0;
     fence_barrier_init();
   }
@@ -648,23 +747,31 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     RingPos pos{0, 0};
     bool ok = true;
     const uint32_t stage_bytes = (uint32_t)kRangeStageBytes * (has_u ? 2u : 1u);
-    uint64_t* last_bar[NS] = {};  // barrier the latest copy into each slot completes on
-    uint32_t last_parity[NS] = {};
-    uint32_t n_stage_copies[NS] = {};  // row stages that have gone through each slot
+    // per slot, as bit masks (arrays indexed by the slot would live in local memory): the parity of the next
+    // row-stage phase of full[slot]; whether the latest copy into the slot was a sample, and that copy's parity
+    uint32_t stage_parity = 0, last_is_sample = 0, last_parity = 0, used = 0;
+    int last_sample_of = 0;
     auto issue = [&](int x, int row, int sample_of) {  // sample_of: -1 for a row stage, else the live row's index
       if (pos.use > 0) ok = mbar_wait_abortable(&sm.empty[pos.slot], (pos.use - 1) & 1u, abort_flag);
       ok = ok && (*abort_flag == 0);
       if (!ok) return;
       unsigned char* dst = sm.ring + (size_t)pos.slot * (2 * kRangeStageBytes);
+      const uint32_t bit = 1u << pos.slot;
       uint64_t* bar;
+      uint32_t parity;
       if (sample_of >= 0) {
         bar = &sm.sample_full[sample_of & 1];
-        last_parity[pos.slot] = ((uint32_t)sample_of >> 1) & 1u;
+        parity = ((uint32_t)sample_of >> 1) & 1u;
+        last_is_sample |= bit;
+        last_sample_of = sample_of;
       } else {
         bar = &sm.full[pos.slot];
-        last_parity[pos.slot] = n_stage_copies[pos.slot]++ & 1u;
+        parity = (stage_parity >> pos.slot) & 1u;
+        stage_parity ^= bit;
+        last_is_sample &= ~bit;
       }
-      last_bar[pos.slot] = bar;
+      last_parity = parity ? (last_parity | bit) : (last_parity & ~bit);
+      used |= bit;
       mbar_arrive_expect_tx(bar, stage_bytes);
       tma_load_box(dst, &map_c, x, row, bar);
       if (has_u) tma_load_box(dst + kRangeStageBytes, &map_u, x, row, bar);
@@ -676,9 +783,16 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       const int row = sm.tab[k].row;
       for (int s = 0; s < cfg.stages && ok; ++s) issue(s * BW, row, -1);
     }
-    // drain: every copy armed here must have landed before the CTA may exit
-    for (int sl = 0; sl < NS; ++sl)
-      if (last_bar[sl] != nullptr) mbar_wait(last_bar[sl], last_parity[sl]);
+    // drain: every copy armed here must have landed before the CTA may exit.  The latest copy into a slot
+    // is the only one that can still be in flight; a slot whose latest copy was a sample holds the latest
+    // sample issued (two samples are at least three copies apart).
+#pragma unroll
+    for (int sl = 0; sl < NS; ++sl) {
+      if ((used >> sl) & 1u) {
+        uint64_t* bar = ((last_is_sample >> sl) & 1u) ? &sm.sample_full[last_sample_of & 1] : &sm.full[sl];
+        mbar_wait(bar, (last_parity >> sl) & 1u);
+      }
+    }
     if (!ok) *abort_flag = 1;
     return;
   }
@@ -722,7 +836,6 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   const int tid = threadIdx.x - NT_F;  // 0 .. NT_P-1
   int flip = 0;
   bool dead = false;
-  float* const pair_vals = reinterpret_cast<float*>(sm.pair_y);  // value 2p + h is half h of pair p
   for (int k = 0; k < n_live; ++k) {
     // from the CTA's last row on, the verification grid may be scheduled (it waits for this grid's end)
     if (k + 1 == n_live) allow_dependent_launch();
@@ -733,8 +846,8 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     RowScratch* rs = a.scratch + row;
     const int kcap = a.kcap;
     // the row's own random number: needed last, computed while waiting
-    const Philox4 rnd = philox4x32_10((uint32_t)re.pos, (uint32_t)(a.seq_base + b), (uint32_t)re.iter, (uint32_t)a.purpose,
-                                      a.seed_lo, a.seed_hi);
+    const uint64_t rnd64 = random64(philox4x32_10((uint32_t)re.pos, (uint32_t)(a.seq_base + b), (uint32_t)re.iter,
+                                                  (uint32_t)a.purpose, a.seed_lo, a.seed_hi));
     if (!dead) dead = !mbar_wait_abortable(sm.cand_full, (uint32_t)k & 1u, abort_flag);
     dead = group_any<NT_P, BAR_P>(dead || (*abort_flag != 0));
     if (dead) {
@@ -750,79 +863,82 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     const float top = __int_as_float(sm.ctl[kRcRowTop]);
     const uint32_t n_pairs = (uint32_t)sm.ctl[kRcRowPairs];
     bool fallback = kcap > kKcapMax || sm.ctl[kRcRowFallback] != 0;
-    if (fallback) {
-      // exact any-shape path from global memory (the row is still in L2); its scratch sits on st_vals, so
-      // that the bins (= st_ids) stay clear
-      group_sync<NT_P, BAR_P>();
-      if (tid == 0) mbar_arrive(sm.cand_free);
-      redo_row<DTYPE, NT_P, BAR_P>(a, row, tid, sm.st_vals);
-      continue;
-    }
-    // ---- every thread takes an equal share of the pair list: a run of consecutive pairs, so that
-    // concatenating the threads' survivors keeps the id order.  Linear bins over [tau0, top] (top: the largest
-    // sample value; anything above it lands in the last bin); monotone in y, so a higher bin never holds a
-    // smaller value.  A thread keeps the bins of its values in registers: 0 = below tau0 (not a candidate),
-    // otherwise bin + 1.
-    const float range = __fsub_rn(top, tau0);
-    const float scale = range > 0.0f ? __fdiv_rn((float)kSelBins * 0.999f, range) : 0.0f;
-    const uint32_t chunk = (n_pairs + NT_P - 1) / NT_P;  // <= kPairChunk
+    // ---- every thread takes an equal share of the pair list into registers: a run of consecutive pairs, so
+    // that concatenating the threads' survivors keeps the id order.  The list then goes straight back to the
+    // filter warps, which may already be waiting to write the next row's.
+    const uint32_t chunk = fallback ? 0u : (n_pairs + NT_P - 1) / NT_P;  // <= kPairChunk
     const uint32_t my_first = min((uint32_t)tid * chunk, n_pairs);
-    const uint32_t my_count = min(my_first + chunk, n_pairs) - my_first;
+    const uint32_t my_count = fallback ? 0u : min(my_first + chunk, n_pairs) - my_first;
+    float2 v[kPairChunk];
+    uint32_t qq[(kPairChunk + 1) / 2];  // pair numbers, two to a word
+#pragma unroll
+    for (int j = 0; j < kPairChunk; ++j) {
+      // a slot beyond the thread's share reads a valid address and is masked out below
+      const uint32_t at = min(my_first + (uint32_t)j, (uint32_t)kRangePairCap - 1u);
+      v[j] = *reinterpret_cast<const float2*>(&sm.pair_y[at]);
+      const uint32_t q = sm.pair_q[at];
+      if ((j & 1) == 0) qq[j >> 1] = q;
+      else qq[j >> 1] |= q << 16;
+    }
     if (tid == 0) {
       sm.ctl[kRcGather] = 0;
       sm.ctl[kRcPtok] = 0;
       sm.ctl[kRcFoundId] = -1;
     }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(sm.cand_free);
+    if (fallback) {
+      if (tid == 0) sm.redo[sm.ctl[kRcRedo]++] = row;  // redone by the any-shape path after the last row
+      continue;
+    }
+    // ---- linear bins over [tau0, top] (top: the largest sample value; anything above it lands in the last
+    // bin); monotone in y, so a higher bin never holds a smaller value.  A thread keeps the bins of its values
+    // in registers: 0 = below tau0 (not a candidate), otherwise bin + 1.
+    const float range = __fsub_rn(top, tau0);
+    const float scale = range > 0.0f ? __fdiv_rn((float)kSelBins * 0.999f, range) : 0.0f;
     uint32_t code[kPairChunk];
     float vmax = neg_inf;
-    constexpr int kHalf = (kPairChunk + 1) / 2;  // loads in flight together
 #pragma unroll
-    for (int j0 = 0; j0 < kPairChunk; j0 += kHalf) {
-      // loads first (a slot beyond the thread's share reads a valid address and is masked out)
-      float2 v[kHalf];
-#pragma unroll
-      for (int u = 0; u < kHalf; ++u)
-        if (j0 + u < kPairChunk)
-          v[u] = *reinterpret_cast<const float2*>(&sm.pair_y[min(my_first + (uint32_t)(j0 + u), (uint32_t)kRangePairCap - 1u)]);
-#pragma unroll
-      for (int u = 0; u < kHalf; ++u) {
-        if (j0 + u < kPairChunk) {
-          const bool mine = (uint32_t)(j0 + u) < my_count;
-          const bool v0 = mine && v[u].x >= tau0, v1 = mine && v[u].y >= tau0;  // false for NaN
-          const int q0 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[u].x, tau0), scale)), kSelBins - 1);
-          const int q1 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[u].y, tau0), scale)), kSelBins - 1);
-          const uint32_t c0 = v0 ? (uint32_t)q0 + 1u : 0u, c1 = v1 ? (uint32_t)q1 + 1u : 0u;
-          code[j0 + u] = c0 | (c1 << 16);
-          vmax = fmaxf(vmax, v0 ? v[u].x : neg_inf);
-          vmax = fmaxf(vmax, v1 ? v[u].y : neg_inf);
-          if (c0 != 0u) atomicAdd(&sm.sel[c0 - 1u], 1u);
-          if (c1 != 0u) atomicAdd(&sm.sel[c1 - 1u], 1u);
-        }
-      }
+    for (int j = 0; j < kPairChunk; ++j) {
+      const bool mine = (uint32_t)j < my_count;
+      const bool v0 = mine && v[j].x >= tau0, v1 = mine && v[j].y >= tau0;  // false for NaN
+      const int q0 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[j].x, tau0), scale)), kSelBins - 1);
+      const int q1 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[j].y, tau0), scale)), kSelBins - 1);
+      const uint32_t c0 = v0 ? (uint32_t)q0 + 1u : 0u, c1 = v1 ? (uint32_t)q1 + 1u : 0u;
+      code[j] = c0 | (c1 << 16);
+      vmax = fmaxf(vmax, v0 ? v[j].x : neg_inf);
+      vmax = fmaxf(vmax, v1 ? v[j].y : neg_inf);
+      if (c0 != 0u) atomicAdd(&sm.sel[c0 - 1u], 1u);
+      if (c1 != 0u) atomicAdd(&sm.sel[c1 - 1u], 1u);
     }
-    // the row's maximum: per warp here, combined after the barriers of the search below
+    // the row's maximum: per warp here, combined after the barrier
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, d));
     float* const warp_max = reinterpret_cast<float*>(sm.scan_p + 64);
     if (lane == 0) warp_max[warp - NF] = vmax;
     group_sync<NT_P, BAR_P>();
     SJD_PHASE(17);
-    // ---- exact K-th largest: threshold bin, then ranking inside it by (y descending, id ascending) ----
-    find_rank_bin<kSelBins, NT_P, BAR_P>(sm.sel, (uint32_t)kcap, tid, sm.scan_p, flip, sm.ctl, kRcPBin);
-    const int tbin = sm.ctl[kRcPBin];
-    const int need = kcap - sm.ctl[kRcPAbove];  // members of the threshold bin that survive
-    const int nbin = sm.ctl[kRcPCount];
+    // ---- exact K-th largest: threshold bin, then ranking inside it by (y descending, id ascending).  Every
+    // warp searches the whole histogram for itself (no barrier).
+    int tbin, need, nbin;
+    {
+      const RankBin rb = warp_rank_bin<kSelBins, false>(sm.sel, (uint32_t)kcap, lane);
+      tbin = rb.bin();
+      need = kcap - (int)rb.above;  // members of the threshold bin that survive
+      nbin = (int)rb.count();
+    }
 #pragma unroll
     for (int w = 0; w < NP; ++w) vmax = fmaxf(vmax, warp_max[w]);
     // fewer than kcap candidates (the sampled threshold was too high), a threshold bin too crowded for the
     // on-chip ranking, or no finite maximum: the any-shape path redoes the row
     if (tbin < 0 || nbin > kBinListCap || !(vmax <= 3.402823466e38f)) fallback = true;
     SJD_PHASE(18);
+    const uint32_t tcode = (uint32_t)tbin + 1u;
     uint32_t n_above = 0;
-    bool in_bin = false;
+    uint32_t hits = 0;  // bit 2j + h: value h of pair j lies in the threshold bin
+    int my_at0 = -1, my_at1 = -1;
+    bool many = false;
     if (!fallback) {
-      const uint32_t tcode = (uint32_t)tbin + 1u;
-      uint32_t hits = 0;  // bit 2j + h: value h of pair j lies in the threshold bin
 #pragma unroll
       for (int j = 0; j < kPairChunk; ++j) {
         const uint32_t c0 = code[j] & 0xffffu, c1 = code[j] >> 16;
@@ -830,84 +946,94 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
         hits |= (c0 == tcode ? 1u : 0u) << (2 * j);
         hits |= (c1 == tcode ? 1u : 0u) << (2 * j + 1);
       }
-      in_bin = hits != 0u;
-      while (hits != 0u) {  // a handful of values per row
-        const int bit = __ffs((int)hits) - 1;
-        hits &= hits - 1u;
-        const int slot = (int)(2u * my_first) + bit;
-        sm.binlist[atomicAdd(&sm.ctl[kRcGather], 1)] = BinMember{pair_vals[slot], slot};
+      // the members of the threshold bin (a handful per row) go on a list: value and position in the pair
+      // list; the thread remembers where its first two went
+#pragma unroll
+      for (int j = 0; j < kPairChunk; ++j) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if ((hits >> (2 * j + h)) & 1u) {
+            const int at = atomicAdd(&sm.ctl[kRcGather], 1);
+            sm.binlist[at] = BinMember{h == 0 ? v[j].x : v[j].y, (int)(2u * (my_first + j)) + h};
+            if (my_at0 < 0) my_at0 = at;
+            else if (my_at1 < 0) my_at1 = at;
+            else many = true;
+          }
+        }
       }
     }
     group_sync<NT_P, BAR_P>();
+    // one thread per member ranks it against the list: the `need` best survive (ties to the lower id), the
+    // others are marked (slot made negative)
     if (!fallback) {
-      // losers of the threshold bin are struck from the pair list: their value becomes -inf
       for (int x = tid; x < nbin; x += NT_P) {
         const BinMember me = sm.binlist[x];
         int rank = 0;
         for (int z = 0; z < nbin; ++z) {
           const BinMember o = sm.binlist[z];
-          rank += (o.y > me.y || (o.y == me.y && o.slot < me.slot)) ? 1 : 0;
+          const int o_slot = o.slot < 0 ? -1 - o.slot : o.slot;  // another thread may have marked it already
+          rank += (o.y > me.y || (o.y == me.y && o_slot < me.slot)) ? 1 : 0;
         }
-        if (rank >= need) pair_vals[me.slot] = neg_inf;
+        if (rank >= need) sm.binlist[x].slot = -1 - me.slot;
       }
     }
     group_sync<NT_P, BAR_P>();
+    // every thread strikes its marked members from `hits`
+    if (!fallback && hits != 0u) {
+      const int slot0 = (int)(2u * my_first);
+      if (!many) {
+        if (my_at0 >= 0) {
+          const int sl = sm.binlist[my_at0].slot;
+          if (sl < 0) hits &= ~(1u << (-1 - sl - slot0));
+        }
+        if (my_at1 >= 0) {
+          const int sl = sm.binlist[my_at1].slot;
+          if (sl < 0) hits &= ~(1u << (-1 - sl - slot0));
+        }
+      } else {  // more than two members in one thread's share (many equal values): look through the list
+        for (int x = 0; x < nbin; ++x) {
+          const int sl = sm.binlist[x].slot;
+          const uint32_t rel = (uint32_t)(-1 - sl - slot0);
+          if (sl < 0 && rel < 2u * my_count) hits &= ~(1u << rel);
+        }
+      }
+    }
     SJD_PHASE(19);
-    uint32_t my_alive = n_above;
-    if (in_bin) {
-      const uint32_t tcode = (uint32_t)tbin + 1u;
+    uint32_t total_alive;
+    uint32_t out_pos = group_scan1<NT_P, BAR_P, uint32_t>(n_above + (uint32_t)__popc(hits), tid, sm.scan_p, flip, &total_alive);
+    if (!fallback && total_alive != (uint32_t)kcap) fallback = true;  // cannot happen; keep the result exact anyway
+    if (!fallback) {
+      // ---- survivors, already in ascending id order (this overwrites sel and the member list).  The
+      // position of each follows from the bits of those before it, so the stores do not wait for one another.
+      uint32_t alive = hits;
 #pragma unroll
       for (int j = 0; j < kPairChunk; ++j) {
         const uint32_t c0 = code[j] & 0xffffu, c1 = code[j] >> 16;
-        if (c0 == tcode && pair_vals[2u * (my_first + j)] >= tau0) ++my_alive;
-        if (c1 == tcode && pair_vals[2u * (my_first + j) + 1u] >= tau0) ++my_alive;
+        alive |= (c0 > tcode ? 1u : 0u) << (2 * j);
+        alive |= (c1 > tcode ? 1u : 0u) << (2 * j + 1);
       }
-    }
-    uint32_t total_alive;
-    uint32_t out_pos = group_scan1<NT_P, BAR_P, uint32_t>(my_alive, tid, sm.scan_p, flip, &total_alive);
-    if (!fallback && total_alive != (uint32_t)kcap) fallback = true;  // cannot happen; keep the result exact anyway
-    if (!fallback) {
-      // ---- survivors, already in ascending id order (this overwrites sel and binlist) ----
-      const uint32_t tcode = (uint32_t)tbin + 1u;
 #pragma unroll
-      for (int j0 = 0; j0 < kPairChunk; j0 += kHalf) {
-        float2 v[kHalf];
-        int id[kHalf];
-#pragma unroll
-        for (int u = 0; u < kHalf; ++u) {
-          if (j0 + u < kPairChunk) {
-            const uint32_t at = min(my_first + (uint32_t)(j0 + u), (uint32_t)kRangePairCap - 1u);
-            v[u] = *reinterpret_cast<const float2*>(&sm.pair_y[at]);
-            id[u] = 2 * (int)sm.pair_q[at];
-          }
+      for (int j = 0; j < kPairChunk; ++j) {
+        const int id = 2 * (int)((qq[j >> 1] >> (16 * (j & 1))) & 0xffffu);
+        const uint32_t at0 = out_pos + (uint32_t)__popc(alive & ((1u << (2 * j)) - 1u));
+        const uint32_t at1 = out_pos + (uint32_t)__popc(alive & ((1u << (2 * j + 1)) - 1u));
+        if ((alive >> (2 * j)) & 1u) {
+          sm.st_ids[at0] = id;
+          sm.st_vals[at0] = canonical(v[j].x);
         }
-#pragma unroll
-        for (int u = 0; u < kHalf; ++u) {
-          if (j0 + u < kPairChunk) {
-            const uint32_t c0 = code[j0 + u] & 0xffffu, c1 = code[j0 + u] >> 16;
-            if (c0 > tcode || (c0 == tcode && v[u].x >= tau0)) {
-              sm.st_ids[out_pos] = id[u];
-              sm.st_vals[out_pos] = canonical(v[u].x);
-              ++out_pos;
-            }
-            if (c1 > tcode || (c1 == tcode && v[u].y >= tau0)) {
-              sm.st_ids[out_pos] = id[u] + 1;
-              sm.st_vals[out_pos] = canonical(v[u].y);
-              ++out_pos;
-            }
-          }
+        if ((alive >> (2 * j + 1)) & 1u) {
+          sm.st_ids[at1] = id + 1;
+          sm.st_vals[at1] = canonical(v[j].y);
         }
       }
     }
     group_sync<NT_P, BAR_P>();
     SJD_PHASE(20);
-    // the pair list is not read again: hand it back
-    if (tid == 0) mbar_arrive(sm.cand_free);
     if (fallback) {
-      // exact any-shape path from global memory.  The bins were cleared when they were read; the any-shape
-      // path's scratch sits on st_vals.
+      // redone by the any-shape path after the last row; the bins must be clear again for the next one
       for (int j = tid; j < kSelBins; j += NT_P) sm.sel[j] = 0;
-      redo_row<DTYPE, NT_P, BAR_P>(a, row, tid, sm.st_vals);
+      if (tid == 0) sm.redo[sm.ctl[kRcRedo]++] = row;
+      group_sync<NT_P, BAR_P>();
       continue;
     }
     // ---- normalise, write the row, draw from it ----
@@ -923,8 +1049,8 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       zpart += e[j];
     }
     // these words of st_ids are this thread's share of sel: zero again for the next row
-    *reinterpret_cast<uint4*>(sm.sel + k0) = make_uint4(0u, 0u, 0u, 0u);
-    *reinterpret_cast<uint4*>(sm.sel + k0 + 4) = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int x = 0; x < kFinItems / 4; ++x) *reinterpret_cast<uint4*>(sm.sel + k0 + 4 * x) = make_uint4(0u, 0u, 0u, 0u);
     const float Z = group_sum1_f32<NT_P, BAR_P>(zpart, tid, sm.scan_p, flip);
     SJD_PHASE(21);
     int32_t* out_ids = a.out_ids + (size_t)row * kcap;
@@ -942,10 +1068,11 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     if ((kcap & 3) == 0 && k0 + kFinItems <= kcap) {
       int4* oi = reinterpret_cast<int4*>(out_ids + k0);
       float4* ov = reinterpret_cast<float4*>(out_vals + k0);
-      oi[0] = make_int4(ids[0], ids[1], ids[2], ids[3]);
-      oi[1] = make_int4(ids[4], ids[5], ids[6], ids[7]);
-      ov[0] = make_float4(p[0], p[1], p[2], p[3]);
-      ov[1] = make_float4(p[4], p[5], p[6], p[7]);
+#pragma unroll
+      for (int x = 0; x < kFinItems / 4; ++x) {
+        oi[x] = make_int4(ids[4 * x], ids[4 * x + 1], ids[4 * x + 2], ids[4 * x + 3]);
+        ov[x] = make_float4(p[4 * x], p[4 * x + 1], p[4 * x + 2], p[4 * x + 3]);
+      }
     } else {
 #pragma unroll
       for (int j = 0; j < kFinItems; ++j) {
@@ -959,7 +1086,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     // the row's own draw from p_i: fixed-point inverse CDF in ascending-id order
     uint64_t T;
     const uint64_t lo = group_scan1<NT_P, BAR_P, uint64_t>(wloc, tid, sm.scan_p, flip, &T);
-    const uint64_t t = __umul64hi(random64(rnd), T);
+    const uint64_t t = __umul64hi(rnd64, T);
     if (T > 0 && t >= lo && t < lo + wloc) {
       uint64_t run = lo;
       int j = 0;
@@ -995,6 +1122,13 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     SJD_PHASE_COUNT(40, 1);
     SJD_PHASE_COUNT(41, n_pairs);
   }
+  // ---- rows the single pass could not finish: the exact any-shape path from global memory (rare).  Kept
+  // out of the loop so that the loop holds no call and nothing of it lives across one.  Its scratch sits on
+  // st_vals.
+  group_sync<NT_P, BAR_P>();
+  const int n_redo = dead ? 0 : sm.ctl[kRcRedo];
+  for (int r = 0; r < n_redo; ++r)
+    row_generic<DTYPE, NT_P, BAR_P>(a, sm.redo[r], tid, *reinterpret_cast<GenericSmem*>(sm.st_vals), kRowStatusRedone);
 }
 
 }  // namespace sjd

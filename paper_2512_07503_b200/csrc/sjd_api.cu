@@ -224,16 +224,17 @@ cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&lc, kern, std::forward<Args>(args)...);
 }
 
-constexpr int kSamplerWarps = 4;
+constexpr int kSamplerWarps = 3;
+constexpr int kRangeFinisherWarps = 16;
 
 template <int DTYPE>
 cudaError_t launch_ranges(const sjd::RowArgs& ra, const sjd::RangeCfg& cfg, const CUtensorMap& mc, const CUtensorMap& mu,
                           size_t smem, int grid, cudaStream_t st) {
-  auto kern = sjd::rows_ranges_kernel<DTYPE, kFinisherWarps, kSamplerWarps>;
+  auto kern = sjd::rows_ranges_kernel<DTYPE, kRangeFinisherWarps, kSamplerWarps>;
   static sjd::DeviceOnce configured;  // per instantiation
   const cudaError_t e = allow_large_smem(kern, configured, (int)kSmemLimit);
   if (e != cudaSuccess) return e;
-  return launch_after(kern, dim3((unsigned)grid), dim3((8 + kFinisherWarps + kSamplerWarps + 1) * 32), smem, st, true, ra,
+  return launch_after(kern, dim3((unsigned)grid), dim3((8 + kRangeFinisherWarps + kSamplerWarps + 1) * 32), smem, st, true, ra,
                       cfg, mc, mu);
 }
 
