@@ -85,7 +85,7 @@ enum {
   kRcTau0, kRcTau1, kRcTau2, kRcTau3,                   // tau0 of live row k in word kRcTau0 + (k & 3)
   kRcTop0, kRcTop1, kRcTop2, kRcTop3,                   // largest sample value of live row k, likewise
   kRcRowTau0, kRcRowTop, kRcRowPairs, kRcRowFallback,   // handed over with the row
-  kRcPBin, kRcPAbove, kRcPCount, kRcGather, kRcPtok, kRcFoundId, kRcFoundP, kRcRedo,  // finisher
+  kRcPBin, kRcPAbove, kRcPCount, kRcGather, kRcPtok, kRcFoundId, kRcFoundP, kRcRedo, kRcRndLo, kRcRndHi,  // finisher
   kRcWords = 32
 };
 
@@ -845,9 +845,13 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     const int b = row / a.W;
     RowScratch* rs = a.scratch + row;
     const int kcap = a.kcap;
-    // the row's own random number: needed last, computed while waiting
-    const uint64_t rnd64 = random64(philox4x32_10((uint32_t)re.pos, (uint32_t)(a.seq_base + b), (uint32_t)re.iter,
-                                                  (uint32_t)a.purpose, a.seed_lo, a.seed_hi));
+    // the row's own random number: needed last, computed by one thread while the others wait
+    if (tid == NT_P - 1) {
+      const uint64_t r = random64(philox4x32_10((uint32_t)re.pos, (uint32_t)(a.seq_base + b), (uint32_t)re.iter,
+                                                (uint32_t)a.purpose, a.seed_lo, a.seed_hi));
+      sm.ctl[kRcRndLo] = (int)(uint32_t)r;
+      sm.ctl[kRcRndHi] = (int)(uint32_t)(r >> 32);
+    }
     if (!dead) dead = !mbar_wait_abortable(sm.cand_full, (uint32_t)k & 1u, abort_flag);
     dead = group_any<NT_P, BAR_P>(dead || (*abort_flag != 0));
     if (dead) {
@@ -918,15 +922,20 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     if (lane == 0) warp_max[warp - NF] = vmax;
     group_sync<NT_P, BAR_P>();
     SJD_PHASE(17);
-    // ---- exact K-th largest: threshold bin, then ranking inside it by (y descending, id ascending).  Every
-    // warp searches the whole histogram for itself (no barrier).
-    int tbin, need, nbin;
-    {
+    // ---- exact K-th largest: threshold bin, then ranking inside it by (y descending, id ascending).  One
+    // warp searches the histogram; the others pick the result up behind a barrier.
+    if (warp == NF) {
       const RankBin rb = warp_rank_bin<kSelBins, false>(sm.sel, (uint32_t)kcap, lane);
-      tbin = rb.bin();
-      need = kcap - (int)rb.above;  // members of the threshold bin that survive
-      nbin = (int)rb.count();
+      if (lane == 0) {
+        sm.ctl[kRcPBin] = rb.bin();
+        sm.ctl[kRcPAbove] = (int)rb.above;
+        sm.ctl[kRcPCount] = (int)rb.count();
+      }
     }
+    group_sync<NT_P, BAR_P>();
+    const int tbin = sm.ctl[kRcPBin];
+    const int need = kcap - sm.ctl[kRcPAbove];  // members of the threshold bin that survive
+    const int nbin = sm.ctl[kRcPCount];
 #pragma unroll
     for (int w = 0; w < NP; ++w) vmax = fmaxf(vmax, warp_max[w]);
     // fewer than kcap candidates (the sampled threshold was too high), a threshold bin too crowded for the
@@ -1086,6 +1095,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     // the row's own draw from p_i: fixed-point inverse CDF in ascending-id order
     uint64_t T;
     const uint64_t lo = group_scan1<NT_P, BAR_P, uint64_t>(wloc, tid, sm.scan_p, flip, &T);
+    const uint64_t rnd64 = (uint64_t)(uint32_t)sm.ctl[kRcRndLo] | ((uint64_t)(uint32_t)sm.ctl[kRcRndHi] << 32);
     const uint64_t t = __umul64hi(rnd64, T);
     if (T > 0 && t >= lo && t < lo + wloc) {
       uint64_t run = lo;

@@ -96,7 +96,14 @@ class DecodeLoop:
         self.steps += 1
 
     def done(self) -> bool:
-        return bool((self.win_len == 0).all().item())
+        """True when every sequence is complete.  This is the loop's one synchronisation point per iteration: the
+        status words of the last step come back with it, and a step whose on-chip wait gave up (its outputs are
+        invalid, and the window was advanced on them) raises here instead of passing unnoticed."""
+        state = torch.stack([(self.win_len != 0).any().to(torch.int32),
+                             (self.status & B.SJD_STATUS_INTERNAL_TIMEOUT).any().to(torch.int32)]).cpu()
+        if int(state[1]) != 0:
+            raise B.SjdError("a step reported SJD_STATUS_INTERNAL_TIMEOUT: its outputs are invalid")
+        return int(state[0]) == 0
 
     def run(self, logit_source: Callable[["DecodeLoop"], Tuple[torch.Tensor, Optional[torch.Tensor]]],
             max_steps: Optional[int] = None):

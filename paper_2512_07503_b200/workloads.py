@@ -183,22 +183,46 @@ class MarkovSource:
     only: an unchanged prefix reproduces the same logits in every iteration.  No method arithmetic here."""
 
     def __init__(self, V: int, n_total: int, dtype: int, states: int = 1024, sigma: float = 3.0, seed_table: int = 7,
-                 seed_c: int = 5, seed_u: int = 6):
+                 seed_c: int = 5, seed_u: int = 6, lazy: bool = False):
         self.V, self.N, self.dtype, self.states = V, n_total, dtype, states
         self.table = markov_table(V, states, sigma, seed_table)
-        self.noise_c = np.stack([markov_noise(V, p, seed_c) for p in range(n_total)])
-        self.noise_u = np.stack([markov_noise(V, p, seed_u) for p in range(n_total)])
+        self.seed_c, self.seed_u = seed_c, seed_u
+        # the noise rows: all at once for small problems; drawn when first asked for, and kept while the window
+        # is near, at the decode-loop workload's full size (2 x 2,304 x 65,536 floats would be 1.2 GB)
+        self._rows = {} if lazy else None
+        if not lazy:
+            self.noise_c = np.stack([markov_noise(V, p, seed_c) for p in range(n_total)])
+            self.noise_u = np.stack([markov_noise(V, p, seed_u) for p in range(n_total)])
+        self._last_key, self._last = None, None
+
+    def _noise(self, pos: int):
+        if self._rows is None:
+            return self.noise_c[pos], self.noise_u[pos]
+        hit = self._rows.get(pos)
+        if hit is None:
+            hit = (markov_noise(self.V, pos, self.seed_c), markov_noise(self.V, pos, self.seed_u))
+            self._rows[pos] = hit
+            for old in [q for q in self._rows if q < pos - 256]:  # the window only moves forward
+                del self._rows[old]
+        return hit
 
     def logits(self, drafts: np.ndarray, win_len: np.ndarray, pos_base: np.ndarray, committed: np.ndarray):
         """cond, uncond of shape [B,W,V] in the storage type, for the given window state."""
         B, W = drafts.shape
+        # the same window asked for twice in a row (two decoders in lock-step) is answered from memory
+        key = (drafts.tobytes(), win_len.tobytes(), pos_base.tobytes(),
+               tuple(int(committed[b, int(pos_base[b]) - 1]) if int(pos_base[b]) > 0 else 0 for b in range(B)))
+        if key == self._last_key:
+            return self._last
         cond = np.zeros((B, W, self.V), np.float32)
         unc = np.zeros((B, W, self.V), np.float32)
         for b in range(B):
             p0 = int(pos_base[b])
             for i in range(int(win_len[b])):
                 prev = int(drafts[b, i - 1]) if i > 0 else (int(committed[b, p0 - 1]) if p0 > 0 else 0)
-                c = self.table[prev % self.states] + self.noise_c[p0 + i]
+                nc, nu = self._noise(p0 + i)
+                c = self.table[prev % self.states] + nc
                 cond[b, i] = c
-                unc[b, i] = c + self.noise_u[p0 + i]
-        return _store(cond, self.dtype), _store(unc, self.dtype)
+                unc[b, i] = c + nu
+        self._last_key, self._last = key, (_store(cond, self.dtype), _store(unc, self.dtype))
+        return self._last

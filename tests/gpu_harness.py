@@ -93,7 +93,7 @@ def oracle_prime(inp: wk.StepInputs, n_threads=8) -> oracle.StepResult:
     return oracle.sjd_step(inp.prev_cond, inp.prev_uncond, None, None, V=inp.wl.V, n_threads=n_threads, diag=True, **kw)
 
 
-def check_parity(cond, uncond, drafts, qprobs, kw, win_len, *, expect_flagged_below=0.02, n_threads=8):
+def check_parity(cond, uncond, drafts, qprobs, kw, win_len, *, expect_flagged_below=2e-3, n_threads=8):
     """Run both sides on the same inputs, compare, and return (report, gpu_out, oracle_result)."""
     V = cond.shape[-1]
     ref = oracle.sjd_step(cond, uncond, drafts, qprobs, V=V, n_threads=n_threads, diag=True, **kw)
@@ -105,5 +105,8 @@ def check_parity(cond, uncond, drafts, qprobs, kw, win_len, *, expect_flagged_be
     assert rep.ok(), rep.summary() + "\n" + "\n".join(rep.errors)
     # bit 16 only says that a row took the any-shape path inside the library: no counterpart in the oracle
     assert np.array_equal(got.status & ~16, ref.status), (got.status, ref.status)
-    assert rep.flagged <= max(2, expect_flagged_below * rep.positions), rep.summary()
+    # decisions within 1e-6 of their boundary may fall on either side; they are rare, and rare in every category
+    allowed = max(2, int(expect_flagged_below * rep.positions))
+    for what, n in (("accept", rep.flagged_accept), ("reuse", rep.flagged_reuse), ("sample", rep.flagged_sample)):
+        assert n <= allowed, (what, rep.summary())
     return rep, got, ref

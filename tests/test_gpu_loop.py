@@ -14,9 +14,9 @@ DEV = "cuda:0"
 
 
 def _both(B, W, V, N, top_k, dtype, reuse=True, seed=21, states=64, init_mode=0, grid_width=1, windows=False,
-          use_graphs=False, refine=True):
+          use_graphs=False, refine=True, lazy=False):
     from paper_2512_07503_b200.decode import DecodeLoop
-    src = wk.MarkovSource(V, N, dtype, states=states)
+    src = wk.MarkovSource(V, N, dtype, states=states, lazy=lazy)
     flags = oracle.FLAG_REUSE if reuse else 0
     trace = []
     ref_committed, ref_steps, ref_counts = loop.decode(
@@ -103,3 +103,15 @@ def test_loop_matches_the_oracle(B, W, V, N, K, dtype, reuse):
     assert np.array_equal(got[0], ref[0])
     assert np.all(got[2].sum(axis=0) == N)
     print("steps", got[1], "tokens per step", N * B / max(1, got[2].shape[0] * B))
+
+
+def test_decode_loop_workload_at_full_size_matches_the_oracle():
+    # the decode-loop configuration as benchmarked: one 48 x 48 grid of 2,304 tokens, V = 65,536, W = 32,
+    # bf16 logits, guidance 3.0, top-K 2,000, random initialisation - every iteration in lock-step with the oracle
+    N = 2304
+    got, ref = _both(1, 32, 65536, N, 2000, wk.BF16, seed=5, states=1024, lazy=True)
+    assert got[1] == ref[1], (got[1], ref[1])
+    assert np.array_equal(got[2], ref[2])
+    assert np.array_equal(got[0], ref[0])
+    assert int(got[2].sum()) == N and np.all(got[0] >= 0)
+    print("cfg5 full size: steps", got[1], "step compression", round(N / got[1], 3))
