@@ -82,6 +82,7 @@ enum {
   kRcAbort = 0,
   kRcLive,                                              // live rows of this CTA (entries of the row table)
   kRcABin, kRcAAbove, kRcACount, kRcSmaxKey,           // sampler
+  kRcBBin, kRcBSmaxKey,                                 // the first row's sampling, done by the finisher warps
   kRcTau0, kRcTau1, kRcTau2, kRcTau3,                   // tau0 of live row k in word kRcTau0 + (k & 3)
   kRcTop0, kRcTop1, kRcTop2, kRcTop3,                   // largest sample value of live row k, likewise
   kRcRowTau0, kRcRowTop, kRcRowPairs, kRcRowFallback,   // handed over with the row
@@ -364,10 +365,16 @@ struct StageReader {
 // candidates the filter keeps (the result is exact whatever it is; too few candidates send the row to the
 // any-shape path), so neither the rounding to 11 bits nor the translation of the rank costs exactness.
 // Sampler thread t looks after ranges t, t + NT, t + 2 NT, ... (NT sampler threads; the last round may be short).
-template <int DTYPE, bool HAS_U, bool HAS_T, bool BY_GROUPS, int NA>
+//
+// FIRST = true is the same work done once, for the CTA's first row, by the finisher warps (which have nothing
+// to do yet): many more threads, so the first threshold - which the whole CTA waits for - comes sooner; the
+// sampler warps proper (FIRST = false) start on the second row at the same time.  The two work side by
+// side, so the first-row instance has a histogram (the finisher's bins) and control words of its own.
+template <int DTYPE, bool HAS_U, bool HAS_T, bool BY_GROUPS, int NA, int BAR_A, bool FIRST>
 __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const RangeCfg& cfg, const RangeSmem& sm, int tid) {
   constexpr int NT_A = NA * 32;
-  constexpr int BAR_A = 3;
+  constexpr int kBin = FIRST ? kRcBBin : kRcABin, kSmaxKey = FIRST ? kRcBSmaxKey : kRcSmaxKey;
+  uint32_t* const hist = FIRST ? sm.sel : sm.hist;
   constexpr int TI = DTYPE != 0 ? 4 : 2;                     // groups of eight elements per range in stage 0
   constexpr int NR = (kRangeThreads + NT_A - 1) / NT_A;       // ranges per sampler thread (at most)
   constexpr int NG = NR * TI;                                 // groups per sampler thread (at most)
@@ -380,7 +387,8 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
   const uint32_t n_live = (uint32_t)sm.ctl[kRcLive];
   const uint32_t rank = (uint32_t)(BY_GROUPS ? cfg.group_rank : cfg.sample_rank);
   RingPos pos{0, 0};
-  for (uint32_t k = 0; k < n_live; ++k) {  // live rows of this CTA
+  if (!FIRST) pos.step();  // the second row's sample is the CTA's second copy
+  for (uint32_t k = FIRST ? 0u : 1u; k < (FIRST ? min(n_live, 1u) : n_live); ++k) {  // live rows of this CTA
     SJD_PHASE_BEGIN();
     // ---------------- the sample into registers; first pass on the way: maxima of groups of eight, by key ----------------
     const bool ok = mbar_wait_abortable(&sm.sample_full[k & 1u], (k >> 1) & 1u, abort_flag);
@@ -388,8 +396,11 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
     __half2 cache[BY_GROUPS ? 1 : NG * 4];
     float gmax[NG];
     float smax = neg_inf;
+    // (rounds in which none of a warp's threads has a range leave their entries as they are: nothing)
 #pragma unroll
     for (int g = 0; g < NG; ++g) gmax[g] = neg_inf;
+#pragma unroll
+    for (int x = 0; x < (BY_GROUPS ? 1 : NG * 4); ++x) cache[x] = __floats2half2_rn(neg_inf, neg_inf);
     if (ok) {
       const uint32_t stage0 = ring_addr + (uint32_t)pos.slot * (2 * kRangeStageBytes);
       // one group of eight per round.  The loop is kept rolled (the code of all roles has to stay in the
@@ -397,6 +408,7 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
 #pragma unroll 1
       for (int g = 0; g < NG; ++g) {
         const int r = g / TI, j = g % TI;
+        if (warp_a * 32 + r * NT_A >= kRangeThreads) continue;  // none of this warp's threads has a range in this round
         // a thread without a range in the last round works on a copy of range 255 and counts nothing (the
         // warp stays together for the vote below)
         const bool have = tid + r * NT_A < kRangeThreads;
@@ -423,27 +435,32 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
         if (!BY_GROUPS && cfg.sample_all) {
           if (have) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) atomicAdd(&sm.hist[float_key(y[q]) >> kSampleKeyShift], 1u);
+            for (int q = 0; q < 8; ++q) atomicAdd(&hist[float_key(y[q]) >> kSampleKeyShift], 1u);
           }
         } else {
           // group maxima crowd into a few coarse bins: one atomic per distinct bin of the warp (a thread
           // without a range votes for a bin of its own kind and adds nothing)
           const uint32_t bin = have ? float_key(m8) >> kSampleKeyShift : 0xffffffffu;
           const uint32_t peers = __match_any_sync(0xffffffffu, bin);
-          if (have && (peers & ((1u << lane) - 1u)) == 0u) atomicAdd(&sm.hist[bin], (uint32_t)__popc(peers));
+          if (have && (peers & ((1u << lane) - 1u)) == 0u) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
         }
         smax = fmaxf(smax, m8);
       }
     }
-    __syncwarp();
-    if (lane == 0) {
-      // the slot's barrier counts eight warps: the sampler's share them out
-      const int share = 8 / NA + (warp_a < 8 % NA ? 1 : 0);
-      mbar_arrive(&sm.empty[pos.slot], (uint32_t)share);
+    if (NA <= 8) {
+      __syncwarp();
+      if (lane == 0) {
+        // the slot's barrier counts eight warps: the sampler's share them out
+        const int share = 8 / NA + (warp_a < 8 % NA ? 1 : 0);
+        mbar_arrive(&sm.empty[pos.slot], (uint32_t)share);
+      }
+    } else {
+      group_sync<NT_A, BAR_A>();
+      if (tid == 0) mbar_arrive(&sm.empty[pos.slot], 8u);
     }
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, d));
-    if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(&sm.ctl[kRcSmaxKey]), float_key(smax));
+    if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(&sm.ctl[kSmaxKey]), float_key(smax));
     if (group_any<NT_A, BAR_A>(!ok)) {
       if (tid == 0) *abort_flag = 1;
       return;
@@ -452,15 +469,15 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
     // at least `rank` group maxima (or, binning everything, elements) are >= the lower edge of this bin.  One
     // warp searches and clears the histogram; the others wait.
     if (warp_a == 0) {
-      const RankBin rb = warp_rank_bin<kSampleBins, true>(sm.hist, rank, lane);
-      if (lane == 0) sm.ctl[kRcABin] = rb.bin();
+      const RankBin rb = warp_rank_bin<kSampleBins, true>(hist, rank, lane);
+      if (lane == 0) sm.ctl[kBin] = rb.bin();
     }
     group_sync<NT_A, BAR_A>();
     SJD_PHASE(2);
-    const int cbin = sm.ctl[kRcABin];
+    const int cbin = sm.ctl[kBin];
     float floor_y = cbin >= 0 ? key_float((uint32_t)cbin << kSampleKeyShift) : lowest;
     if (!(floor_y >= lowest)) floor_y = lowest;  // edge fell on -inf or into the NaN patterns
-    const float top_y = key_float((uint32_t)sm.ctl[kRcSmaxKey]);
+    const float top_y = key_float((uint32_t)sm.ctl[kSmaxKey]);
     const bool refine = floor_y > lowest && top_y >= floor_y && top_y <= 3.402823466e38f;
     const float range = __fsub_rn(top_y, floor_y);
     const float scale = (refine && range > 0.0f) ? __fdiv_rn((float)kSampleBins - 0.5f, range) : 0.0f;
@@ -471,7 +488,7 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
           const int bin = min(max(__float2int_rd(__fmul_rn(__fsub_rn(gmax[g], floor_y), scale)), 0), kSampleBins - 1);
-          if (gmax[g] >= floor_y) atomicAdd(&sm.hist[bin], 1u);
+          if (gmax[g] >= floor_y) atomicAdd(&hist[bin], 1u);
         }
       } else {
 #pragma unroll
@@ -479,14 +496,14 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
           const float2 v = __half22float2(cache[j]);
           const int b0 = min(max(__float2int_rd(__fmul_rn(__fsub_rn(v.x, floor_y), scale)), 0), kSampleBins - 1);
           const int b1 = min(max(__float2int_rd(__fmul_rn(__fsub_rn(v.y, floor_y), scale)), 0), kSampleBins - 1);
-          if (v.x >= floor_y) atomicAdd(&sm.hist[b0], 1u);
-          if (v.y >= floor_y) atomicAdd(&sm.hist[b1], 1u);
+          if (v.x >= floor_y) atomicAdd(&hist[b0], 1u);
+          if (v.y >= floor_y) atomicAdd(&hist[b1], 1u);
         }
       }
       group_sync<NT_A, BAR_A>();
       SJD_PHASE(3);
       if (warp_a == 0) {
-        const int fbin = warp_rank_bin<kSampleBins, true>(sm.hist, rank, lane).bin();
+        const int fbin = warp_rank_bin<kSampleBins, true>(hist, rank, lane).bin();
         if (fbin > 0 && scale > 0.0f) {
           // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
           const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
@@ -501,16 +518,38 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
     // a word of its own for each of four consecutive rows: the filter reads it at the start of the row, and
     // the ring keeps the sampler less than two rows ahead of the filter
     if (tid == 0) {
-      sm.ctl[kRcSmaxKey] = 0;  // every thread has read it (barrier above)
+      sm.ctl[kSmaxKey] = 0;  // every thread has read it (barrier above)
       sm.ctl[kRcTau0 + (int)(k & 3u)] = __float_as_int(tau0);
       sm.ctl[kRcTop0 + (int)(k & 3u)] = __float_as_int(top_y);
       mbar_arrive(&sm.tau_full[k & 1u]);
     }
     group_sync<NT_A, BAR_A>();  // the histogram is clear and kRcSmaxKey reset before the next row's first pass
     SJD_PHASE(4);
-    // sample(1) follows sample(0) directly; sample(k+1) follows sample(k) after the S stages of row k-1 and itself
-    if (k == 0) pos.step();
-    else pos.skip(1 + cfg.stages);
+    // sample(k+1) follows sample(k) after the S stages of row k-1 and itself (k >= 1)
+    pos.skip(1 + cfg.stages);
+  }
+}
+
+// the instance of the sampler for this call's arguments
+template <int DTYPE, int NA, int BAR_A, bool FIRST>
+__device__ __forceinline__ void sample_rows(const RowArgs& a, const RangeCfg& cfg, const RangeSmem& sm, int tid, bool has_u,
+                                            bool has_t) {
+  if (cfg.group_rank > 0) {
+    if (has_u) {
+      if (has_t) range_sampler_role<DTYPE, true, true, true, NA, BAR_A, FIRST>(a, cfg, sm, tid);
+      else range_sampler_role<DTYPE, true, false, true, NA, BAR_A, FIRST>(a, cfg, sm, tid);
+    } else {
+      if (has_t) range_sampler_role<DTYPE, false, true, true, NA, BAR_A, FIRST>(a, cfg, sm, tid);
+      else range_sampler_role<DTYPE, false, false, true, NA, BAR_A, FIRST>(a, cfg, sm, tid);
+    }
+  } else {
+    if (has_u) {
+      if (has_t) range_sampler_role<DTYPE, true, true, false, NA, BAR_A, FIRST>(a, cfg, sm, tid);
+      else range_sampler_role<DTYPE, true, false, false, NA, BAR_A, FIRST>(a, cfg, sm, tid);
+    } else {
+      if (has_t) range_sampler_role<DTYPE, false, true, false, NA, BAR_A, FIRST>(a, cfg, sm, tid);
+      else range_sampler_role<DTYPE, false, false, false, NA, BAR_A, FIRST>(a, cfg, sm, tid);
+    }
   }
 }
 
@@ -811,29 +850,14 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   }
   if (warp >= NF + NP) {
     // ======================================= sampler warps =======================================
-    const int t = threadIdx.x - (NF + NP) * 32;
-    if (cfg.group_rank > 0) {
-      if (has_u) {
-        if (has_t) range_sampler_role<DTYPE, true, true, true, NA>(a, cfg, sm, t);
-        else range_sampler_role<DTYPE, true, false, true, NA>(a, cfg, sm, t);
-      } else {
-        if (has_t) range_sampler_role<DTYPE, false, true, true, NA>(a, cfg, sm, t);
-        else range_sampler_role<DTYPE, false, false, true, NA>(a, cfg, sm, t);
-      }
-    } else {
-      if (has_u) {
-        if (has_t) range_sampler_role<DTYPE, true, true, false, NA>(a, cfg, sm, t);
-        else range_sampler_role<DTYPE, true, false, false, NA>(a, cfg, sm, t);
-      } else {
-        if (has_t) range_sampler_role<DTYPE, false, true, false, NA>(a, cfg, sm, t);
-        else range_sampler_role<DTYPE, false, false, false, NA>(a, cfg, sm, t);
-      }
-    }
+    sample_rows<DTYPE, NA, 3, false>(a, cfg, sm, threadIdx.x - (NF + NP) * 32, has_u, has_t);
     return;
   }
 
   // ======================================= finisher warps =======================================
   const int tid = threadIdx.x - NT_F;  // 0 .. NT_P-1
+  // the first row's threshold, while there is nothing to finish yet
+  sample_rows<DTYPE, NP, BAR_P, true>(a, cfg, sm, tid, has_u, has_t);
   int flip = 0;
   bool dead = false;
   for (int k = 0; k < n_live; ++k) {
