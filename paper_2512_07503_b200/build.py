@@ -38,6 +38,9 @@ def is_stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    override = os.environ.get("SJD_LIBRARY")
+    if override:  # a library built elsewhere (the tests build variants with build_variant())
+        return override
     if not force and not is_stale():
         return LIB_PATH
     tmp = LIB_PATH + f".tmp{os.getpid()}"
@@ -45,6 +48,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
+
+
+def build_variant(out_path: str, defines) -> str:
+    """The library with extra -D definitions (test builds: short wait limits, a dropped copy), written to
+    `out_path`.  Load it in a process of its own by setting SJD_LIBRARY to that path."""
+    cmd = [_nvcc(), *NVCC_FLAGS, "-I", _INC, *[f"-D{d}" for d in defines], *sources(), "-o", out_path]
+    subprocess.check_call(cmd)
+    return out_path
 
 
 if __name__ == "__main__":

@@ -46,7 +46,12 @@ constexpr int kBinListCap = 512;          // members of the threshold bin ranked
 constexpr int kKcapMax = 2048;            // largest kcap the on-chip path stages
 constexpr int kFinItems = 8;              // staged entries per finisher thread (kKcapMax / finisher threads)
 constexpr uint32_t kSpinLimit = 1u << 22; // polls before a wait gives up
+#ifdef SJD_TEST_SPIN_CYCLES
+// test builds only: a short limit, so that a test can watch a wait run out (see SJD_TEST_DROP_COPY)
+constexpr long long kSpinCycles = SJD_TEST_SPIN_CYCLES;
+#else
 constexpr long long kSpinCycles = 1ll << 31;  // ... or this many clock cycles, whichever comes first
+#endif
 
 struct PipeCfg {
   int sample_stride;  // SS: every SS-th tile of a row is a sample tile

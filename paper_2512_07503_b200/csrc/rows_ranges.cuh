@@ -811,6 +811,15 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       }
       last_parity = parity ? (last_parity | bit) : (last_parity & ~bit);
       used |= bit;
+#ifdef SJD_TEST_DROP_COPY
+      // test builds only: the CTA's copy number SJD_TEST_DROP_COPY is never issued, so that the wait for it
+      // runs out and the time-out path (status instead of a hang) can be watched
+      if ((int)(pos.use * NS + pos.slot) == SJD_TEST_DROP_COPY) {
+        used &= ~bit;
+        pos.step();
+        return;
+      }
+#endif
       mbar_arrive_expect_tx(bar, stage_bytes);
       tma_load_box(dst, &map_c, x, row, bar);
       if (has_u) tma_load_box(dst + kRangeStageBytes, &map_u, x, row, bar);
