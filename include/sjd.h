@@ -183,17 +183,20 @@ int sjd_row_kernel(const sjd_params* params);
  *                  valid row.  After the caller shifts the window it is a valid draft_probs for the next
  *                  iteration.  Must not alias draft_probs or the logits.
  *
- * Asynchronous on params->stream.  Returns SJD_OK once the kernels are enqueued, or a negative SJD_ERR_*
- * with nothing enqueued.  Conditions found on the device (status bits) never abort the kernels.
+ * Asynchronous on params->stream.  Returns SJD_OK once the kernels are enqueued.  A negative SJD_ERR_* for a
+ * bad argument means that nothing was enqueued; SJD_ERR_CUDA (a launch or an event record refused by the
+ * runtime) may leave the work enqueued before the failing call on the stream.  Conditions found on the
+ * device (status bits) never abort the kernels.  A problem of more than 32 rows per SM takes several launches
+ * of the row kernel.
  */
 int sjd_step(const void* logits_cond, const void* logits_uncond, const int32_t* drafts,
              const sjd_probs* draft_probs, const sjd_params* params, uint64_t philox_seed,
              int32_t* out_accept_len, int32_t* out_tokens, sjd_probs* out_probs);
 
 /*
- * Window bookkeeping of the decode loop (Section 4.1: Step 1 "draft token preparation", the last sentence
- * of Step 3 "accepted tokens are appended", the last sentence of Step 4 "accepted and reinitialised tokens
- * form the next window"; random initialisation is the baseline of Section 4.2).
+ * Window bookkeeping of the decode loop (Section 4.1: the preparation of the draft tokens in Step 1, the
+ * commit of the verified tokens at the end of Step 3, the make-up of the next window at the end of Step 4;
+ * random initialisation is the baseline of Section 4.2).
  *
  * sjd_window_init() fills the first window.  With SJD_INIT_RANDOM drafts[b,i] for i < win_len[b] is a token
  * drawn uniformly from [0,V) (Philox purpose 4, counter = (pos_base[b]+i, seq_base+b, iteration[b], 4), token =

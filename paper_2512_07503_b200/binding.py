@@ -196,16 +196,22 @@ def sjd_workspace_bytes(params: sjd_params) -> int:
     return int(lib().sjd_workspace_bytes(C.byref(params)))
 
 
-def sjd_step(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor], drafts: Optional[torch.Tensor],
-             draft_probs: Optional[DeviceProbs], params: sjd_params, philox_seed: int, out_accept_len: torch.Tensor,
-             out_tokens: torch.Tensor, out_probs: DeviceProbs) -> None:
-    """Enqueue one verify-and-redraft step on ``params.stream``.  Same arguments as the C entry point."""
+def _check_logits(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor]) -> None:
+    """What both device entry points ask of the two logits tensors (the C side sees only pointers)."""
     if not logits_cond.is_cuda:
         raise SjdError("logits must live on a CUDA device")
     if logits_uncond is not None and (logits_uncond.shape != logits_cond.shape or
                                       logits_uncond.stride() != logits_cond.stride() or
-                                      logits_uncond.dtype != logits_cond.dtype):
-        raise SjdError("cond and uncond logits must share shape, strides and dtype")
+                                      logits_uncond.dtype != logits_cond.dtype or
+                                      logits_uncond.device != logits_cond.device):
+        raise SjdError("cond and uncond logits must share shape, strides, dtype and device")
+
+
+def sjd_step(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Tensor], drafts: Optional[torch.Tensor],
+             draft_probs: Optional[DeviceProbs], params: sjd_params, philox_seed: int, out_accept_len: torch.Tensor,
+             out_tokens: torch.Tensor, out_probs: DeviceProbs) -> None:
+    """Enqueue one verify-and-redraft step on ``params.stream``.  Same arguments as the C entry point."""
+    _check_logits(logits_cond, logits_uncond)
     q = draft_probs.c_struct() if draft_probs is not None else None
     o = out_probs.c_struct()
     with torch.cuda.device(logits_cond.device):
@@ -252,8 +258,7 @@ def sjd_step_static(logits_cond: torch.Tensor, logits_uncond: Optional[torch.Ten
     they call the library (a frozen allocator, a pool they do not own).  The scratch is a fixed array inside
     the library, good for B*W <= SJD_STATIC_MAX_ROWS; larger problems raise.  ``params.workspace`` is ignored.
     Calls on one device share that array: do not let two of them overlap on the GPU."""
-    if not logits_cond.is_cuda:
-        raise SjdError("logits must live on a CUDA device")
+    _check_logits(logits_cond, logits_uncond)
     q = draft_probs.c_struct() if draft_probs is not None else None
     o = out_probs.c_struct()
     with torch.cuda.device(logits_cond.device):

@@ -3,8 +3,9 @@
 ``sjd_step_static`` exists for hosts that may not allocate device memory where they call the library (an
 allocator frozen after start-up, a memory pool owned by someone else): it takes its scratch from a fixed
 array inside the library instead of a caller-supplied workspace.  It runs the same kernels, so every
-output must equal ``sjd_step``'s bit for bit; two calls in a row check that what the first call left in
-the shared array does not leak into the second.  This file sorts last on purpose: a run that stops at
+output must equal ``sjd_step``'s bit for bit (and, like it, agree with the CPU oracle); two calls in a row
+check that what the first call left in the shared array does not leak into the second.  This file sorts
+last on purpose: a run that stops at
 the first failure has then already run every other test.
 """
 import numpy as np
@@ -12,6 +13,7 @@ import pytest
 import torch
 
 import oracle
+from oracle import compare
 import paper_2512_07503_b200 as sjd
 from paper_2512_07503_b200 import workloads as wk
 
@@ -32,8 +34,12 @@ def _device_inputs(wl):
 
     q = sjd.DeviceProbs(*(torch.from_numpy(a).to(DEV) for a in (prev.probs.tok_prob, prev.probs.ids, prev.probs.vals,
                                                                 prev.probs.cnt)))
+    # what the oracle makes of the same step, for the comparison with the allocation-free entry point
+    ref = oracle.sjd_step(inp.cond, inp.uncond, prev.tokens, prev.probs, flags=oracle.FLAG_REUSE, iteration0=1,
+                          reuse_tau=wl.reuse_tau, diag=True, **kw)
     return dict(cond=up(inp.cond), uncond=up(inp.uncond), drafts=torch.from_numpy(prev.tokens).to(DEV), q=q,
-                win_len=torch.from_numpy(inp.win_len).to(DEV), pos_base=torch.from_numpy(inp.pos_base).to(DEV))
+                win_len=torch.from_numpy(inp.win_len).to(DEV), pos_base=torch.from_numpy(inp.pos_base).to(DEV),
+                ref=ref, host_drafts=prev.tokens, host_win_len=inp.win_len)
 
 
 def _run(entry, wl, d, with_workspace):
@@ -65,6 +71,10 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
         for a, b in zip(got, want):
             assert a.tobytes() == b.tobytes()
         assert (got[0] >= 0).all() and (got[0] <= wl.W).all()
+        acc, toks, flags, status, tok_prob, ids, vals, cnt = got
+        rep = compare.compare_step(acc, toks, tok_prob, flags, ids, vals, cnt, d["ref"], d["host_drafts"],
+                                   d["host_win_len"], oracle.FLAG_REUSE)
+        assert rep.ok(), rep.summary() + "\n" + "\n".join(rep.errors)
 
 
 def test_static_scratch_refuses_what_does_not_fit():
