@@ -87,6 +87,7 @@ enum {
   kRcTop0, kRcTop1, kRcTop2, kRcTop3,                   // largest sample value of live row k, likewise
   kRcRowTau0, kRcRowTop, kRcRowPairs, kRcRowFallback,   // handed over with the row
   kRcPBin, kRcPAbove, kRcPCount, kRcGather, kRcPtok, kRcFoundId, kRcFoundP, kRcRedo, kRcRndLo, kRcRndHi,  // finisher
+  kRcTrashA, kRcTrashB,                                 // where the histogram updates of lanes with nothing to count go
   kRcWords = 32
 };
 
@@ -113,6 +114,8 @@ struct RangeSmem {
   uint32_t* sel;        // [kSelBins]  = st_ids: dead before the survivors are staged
   BinMember* binlist;   // [kBinListCap] = st_vals: likewise
   uint32_t* hist;       // [kSampleBins] sampler
+  uint32_t* hist_c;     // [kSampleBins / 32] its coarse level
+  uint32_t* sel_c;      // [kSelBins / 32] coarse level of sel (and of the first row's sampling, which borrows sel)
   RowEntry* tab;        // [kRowsPerCta]
   int32_t* redo;        // [kRowsPerCta] rows the single pass could not finish (redone at the end)
   uint64_t* full;       // [kRangeRingStages] a row stage has landed in the slot (waited for by the filter)
@@ -138,6 +141,7 @@ __host__ __device__ inline size_t range_smem_bytes(int mask_words) {
   b += (size_t)kRowsPerCta * sizeof(RowEntry);
   b += (size_t)kRowsPerCta * 4;
   b += 16 * 8 + 3 * (2 * 32 + 8) * 8 + kRcWords * 4;
+  b += (size_t)(kSampleBins / 32 + kSelBins / 32) * 4;
   return b;
 }
 
@@ -183,6 +187,9 @@ __device__ __forceinline__ RangeSmem carve_range_smem(unsigned char* base, int m
   s.scan_a = reinterpret_cast<uint64_t*>(p);
   p += (2 * 32 + 8) * 8;
   s.ctl = reinterpret_cast<int*>(p);
+  p += kRcWords * 4;
+  s.hist_c = reinterpret_cast<uint32_t*>(p);
+  s.sel_c = s.hist_c + kSampleBins / 32;
   return s;
 }
 
@@ -246,83 +253,76 @@ __device__ __forceinline__ void tma_load_box(void* dst, const CUtensorMap* map, 
       : "memory");
 }
 
-// Largest bin b with (entries in bins > b) < target <= (entries in bins >= b), found by ONE warp without a
-// barrier: lane l sums bins [P (31 - l), P (32 - l)) with P = BINS / 32, a scan over the lanes finds the lane
-// whose bins hold the rank, and that lane's P bins are spread over the lanes for a second scan.  Every lane
-// gets the result: bin + 1 in bits 0-11 of one word (0 when the histogram holds fewer than `target`
-// entries) with the bin's own count in bits 12-31, and the count above the bin.  Counts stay below 2^20 (a
-// row has at most 2^17 values).  With ZERO the warp also clears the histogram (it must be the only reader).
-// Inlined on purpose, like everything on the roles' paths: an out-of-line function saves and restores
-// registers through local memory, and local memory lies behind the ring's outstanding copies.
+// Histograms come in two levels: BINS fine bins and BINS / 32 coarse ones, coarse[c] counting what fine bins
+// 32 c .. 32 c + 31 count (whoever adds to a fine bin adds to its coarse bin as well: shared-memory atomics
+// that ask for no old value are cheap, a long search by one warp while the others wait is not).
+//
+// rank search: the largest bin b with (entries in bins > b) < target <= (entries in bins >= b), found by one
+// warp with two short scans: over the coarse bins (lane 0 takes the topmost), then over the 32 fine bins of
+// the coarse bin that holds the rank.  Every lane gets the result: bin + 1 in bits 0-11 of one word (0 when
+// the histogram holds fewer than `target` entries) with the bin's own count in bits 12-31, and the count
+// above the bin.  Counts stay below 2^20 (a row has at most 2^17 values).  With ZERO the warp also clears both
+// levels (it must be the only reader).  Inlined on purpose, like everything on the roles' paths: an
+// out-of-line function saves and restores registers through local memory, and local memory lies behind the
+// ring's outstanding copies.
 struct RankBin {
   uint32_t bin_count;  // (count << 12) | (bin + 1)
   uint32_t above;
   __device__ __forceinline__ int bin() const { return (int)(bin_count & 0xfffu) - 1; }
   __device__ __forceinline__ uint32_t count() const { return bin_count >> 12; }
 };
-template <int BINS, bool ZERO>
-__device__ __forceinline__ uint2 warp_rank_bin_raw(uint32_t* hist, uint32_t target, int lane) {
-  constexpr int P = BINS / 32;   // bins per lane
-  constexpr int Q = P / 32;      // bins per lane of the second step
-  static_assert(BINS % 1024 == 0 && (Q == 1 || Q == 2), "1024 or 2048 bins");
-  // a lane's bins lie P words apart from its neighbour's, i.e. in the same banks: every lane starts its walk
-  // at a different 16-byte piece, so that the eight lanes served together touch eight different bank groups
-  uint4* mine = reinterpret_cast<uint4*>(hist + P * (31 - lane));
-  uint32_t sum = 0;
-#pragma unroll
-  for (int x = 0; x < P / 4; ++x) {
-    const uint4 w = mine[(x + lane) & (P / 4 - 1)];
-    sum += w.x + w.y + w.z + w.w;
-  }
-  uint32_t inc = sum;
+__device__ __forceinline__ uint32_t warp_scan_incl(uint32_t v, int lane) {
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
-    const uint32_t n = __shfl_up_sync(0xffffffffu, inc, d);
-    if (lane >= d) inc += n;
+    const uint32_t n = __shfl_up_sync(0xffffffffu, v, d);
+    if (lane >= d) v += n;
   }
-  const uint32_t owner_votes = __ballot_sync(0xffffffffu, inc - sum < target && target <= inc);
-  uint2 result = make_uint2(0u, 0u);
-  if (owner_votes != 0u) {
-    const int owner = __ffs((int)owner_votes) - 1;
-    const uint32_t above0 = __shfl_sync(0xffffffffu, inc - sum, owner);  // entries in bins above the owner's
-    const int seg = P * (31 - owner);                                     // the owner's bins: [seg, seg + P)
-    // lane l takes the Q bins ending at seg + P - 1 - Q l (descending with l); c_hi is the upper one
-    uint32_t c_lo, c_hi;
-    if (Q == 2) {
-      const uint2 c = *reinterpret_cast<const uint2*>(hist + seg + P - 2 - 2 * lane);
-      c_lo = c.x;
-      c_hi = c.y;
-    } else {
-      c_hi = hist[seg + P - 1 - lane];
-      c_lo = 0;
-    }
-    const uint32_t both = c_lo + c_hi;
-    uint32_t inc2 = both;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const uint32_t n = __shfl_up_sync(0xffffffffu, inc2, d);
-      if (lane >= d) inc2 += n;
-    }
-    const uint32_t ab = above0 + inc2 - both;  // above this lane's upper bin
-    const bool in_hi = ab < target && target <= ab + c_hi;
-    const bool in_lo = Q == 2 && ab + c_hi < target && target <= ab + both;
-    const int l2 = __ffs((int)__ballot_sync(0xffffffffu, in_hi || in_lo)) - 1;  // exists: the owner's bins hold the rank
-    const uint32_t my_bin = (uint32_t)(seg + P - Q - Q * lane + ((Q == 2 && in_hi) ? 1 : 0));
-    const uint32_t my_cnt = in_hi ? c_hi : c_lo;
-    result.x = __shfl_sync(0xffffffffu, (my_cnt << 12) | (my_bin + 1u), l2);
-    result.y = __shfl_sync(0xffffffffu, in_hi ? ab : ab + c_hi, l2);
+  return v;
+}
+template <int BINS, bool ZERO>
+__device__ __forceinline__ RankBin warp_rank_bin(uint32_t* fine, uint32_t* coarse, uint32_t target, int lane) {
+  constexpr int C = BINS / 32;  // coarse bins
+  constexpr int Q = C / 32;     // coarse bins per lane
+  static_assert(BINS % 1024 == 0 && (Q == 1 || Q == 2), "1024 or 2048 bins");
+  // lane l: coarse bins C - 1 - Q l (c_hi) and, with two to a lane, the one below it (c_lo)
+  uint32_t c_hi, c_lo = 0;
+  if (Q == 2) {
+    const uint2 c = *reinterpret_cast<const uint2*>(coarse + C - 2 - 2 * lane);
+    c_lo = c.x;
+    c_hi = c.y;
+  } else {
+    c_hi = coarse[C - 1 - lane];
+  }
+  const uint32_t both = c_lo + c_hi;
+  const uint32_t ab = warp_scan_incl(both, lane) - both;  // entries above this lane's upper coarse bin
+  const bool in_hi = ab < target && target <= ab + c_hi;
+  const bool in_lo = Q == 2 && ab + c_hi < target && target <= ab + both;
+  const uint32_t votes = __ballot_sync(0xffffffffu, in_hi || in_lo);
+  RankBin result{0u, 0u};
+  if (votes != 0u) {
+    const int l1 = __ffs((int)votes) - 1;
+    // the coarse bin that holds the rank, and what lies above it
+    const uint32_t mine = ((uint32_t)(C - 1 - Q * lane - (in_lo ? 1 : 0)) << 20) | (in_hi ? ab : ab + c_hi);
+    const uint32_t got = __shfl_sync(0xffffffffu, mine, l1);
+    const uint32_t cbin = got >> 20, above0 = got & 0xfffffu;
+    const uint32_t f = fine[32u * cbin + 31u - (uint32_t)lane];  // lane 0 takes the topmost of its 32 fine bins
+    const uint32_t ab2 = above0 + warp_scan_incl(f, lane) - f;
+    const int l2 = __ffs((int)__ballot_sync(0xffffffffu, ab2 < target && target <= ab2 + f)) - 1;  // exists
+    result.bin_count = (__shfl_sync(0xffffffffu, f, l2) << 12) | (32u * cbin + 31u - (uint32_t)l2 + 1u);
+    result.above = __shfl_sync(0xffffffffu, ab2, l2);
   }
   if (ZERO) {
     __syncwarp();
+    // a lane's share of the fine bins: BINS / 32 consecutive words; lanes start at different 16-byte pieces
+    // so that the eight lanes served together touch eight different bank groups
+    constexpr int P = BINS / 32;
+    uint4* my = reinterpret_cast<uint4*>(fine + P * lane);
 #pragma unroll
-    for (int x = 0; x < P / 4; ++x) mine[(x + lane) & (P / 4 - 1)] = make_uint4(0u, 0u, 0u, 0u);
+    for (int x = 0; x < P / 4; ++x) my[(x + lane) & (P / 4 - 1)] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int x = 0; x < Q; ++x) coarse[Q * lane + x] = 0u;
   }
   return result;
-}
-template <int BINS, bool ZERO>
-__device__ __forceinline__ RankBin warp_rank_bin(uint32_t* hist, uint32_t target, int lane) {
-  const uint2 r = warp_rank_bin_raw<BINS, ZERO>(hist, target, lane);
-  return RankBin{r.x, r.y};
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -375,6 +375,11 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
   constexpr int NT_A = NA * 32;
   constexpr int kBin = FIRST ? kRcBBin : kRcABin, kSmaxKey = FIRST ? kRcBSmaxKey : kRcSmaxKey;
   uint32_t* const hist = FIRST ? sm.sel : sm.hist;
+  uint32_t* const hist_c = FIRST ? sm.sel_c : sm.hist_c;
+  // An atomic with some lanes switched off runs several times slower than one with all lanes on, and lanes that
+  // hit the same word cost nothing extra when the old value is not asked for: a lane with nothing to count
+  // adds to a word nobody reads.
+  uint32_t* const trash = reinterpret_cast<uint32_t*>(sm.ctl + (FIRST ? kRcTrashB : kRcTrashA));
   constexpr int TI = DTYPE != 0 ? 4 : 2;                     // groups of eight elements per range in stage 0
   constexpr int NR = (kRangeThreads + NT_A - 1) / NT_A;       // ranges per sampler thread (at most)
   constexpr int NG = NR * TI;                                 // groups per sampler thread (at most)
@@ -433,16 +438,17 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
           for (int q = 0; q < 4; ++q) cache[BY_GROUPS ? 0 : q] = __floats2half2_rn(y[2 * q], y[2 * q + 1]);
         }
         if (!BY_GROUPS && cfg.sample_all) {
-          if (have) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) atomicAdd(&hist[float_key(y[q]) >> kSampleKeyShift], 1u);
+          for (int q = 0; q < 8; ++q) {
+            const uint32_t bin = float_key(y[q]) >> kSampleKeyShift;
+            atomicAdd(have ? &hist[bin] : trash, 1u);
+            atomicAdd(have ? &hist_c[bin >> 5] : trash, 1u);
           }
         } else {
-          // group maxima crowd into a few coarse bins: one atomic per distinct bin of the warp (a thread
-          // without a range votes for a bin of its own kind and adds nothing)
-          const uint32_t bin = have ? float_key(m8) >> kSampleKeyShift : 0xffffffffu;
-          const uint32_t peers = __match_any_sync(0xffffffffu, bin);
-          if (have && (peers & ((1u << lane) - 1u)) == 0u) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+          // group maxima crowd into a few coarse bins: lanes that meet in one cost no more than lanes apart
+          const uint32_t bin = float_key(m8) >> kSampleKeyShift;
+          atomicAdd(have ? &hist[bin] : trash, 1u);
+          atomicAdd(have ? &hist_c[bin >> 5] : trash, 1u);
         }
         smax = fmaxf(smax, m8);
       }
@@ -469,7 +475,7 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
     // at least `rank` group maxima (or, binning everything, elements) are >= the lower edge of this bin.  One
     // warp searches and clears the histogram; the others wait.
     if (warp_a == 0) {
-      const RankBin rb = warp_rank_bin<kSampleBins, true>(hist, rank, lane);
+      const RankBin rb = warp_rank_bin<kSampleBins, true>(hist, hist_c, rank, lane);
       if (lane == 0) sm.ctl[kBin] = rb.bin();
     }
     group_sync<NT_A, BAR_A>();
@@ -488,7 +494,8 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
           const int bin = min(max(__float2int_rd(__fmul_rn(__fsub_rn(gmax[g], floor_y), scale)), 0), kSampleBins - 1);
-          if (gmax[g] >= floor_y) atomicAdd(&hist[bin], 1u);
+          atomicAdd(gmax[g] >= floor_y ? &hist[bin] : trash, 1u);
+          atomicAdd(gmax[g] >= floor_y ? &hist_c[bin >> 5] : trash, 1u);
         }
       } else {
 #pragma unroll
@@ -496,14 +503,16 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
           const float2 v = __half22float2(cache[j]);
           const int b0 = min(max(__float2int_rd(__fmul_rn(__fsub_rn(v.x, floor_y), scale)), 0), kSampleBins - 1);
           const int b1 = min(max(__float2int_rd(__fmul_rn(__fsub_rn(v.y, floor_y), scale)), 0), kSampleBins - 1);
-          if (v.x >= floor_y) atomicAdd(&hist[b0], 1u);
-          if (v.y >= floor_y) atomicAdd(&hist[b1], 1u);
+          atomicAdd(v.x >= floor_y ? &hist[b0] : trash, 1u);
+          atomicAdd(v.x >= floor_y ? &hist_c[b0 >> 5] : trash, 1u);
+          atomicAdd(v.y >= floor_y ? &hist[b1] : trash, 1u);
+          atomicAdd(v.y >= floor_y ? &hist_c[b1 >> 5] : trash, 1u);
         }
       }
       group_sync<NT_A, BAR_A>();
       SJD_PHASE(3);
       if (warp_a == 0) {
-        const int fbin = warp_rank_bin<kSampleBins, true>(hist, rank, lane).bin();
+        const int fbin = warp_rank_bin<kSampleBins, true>(hist, hist_c, rank, lane).bin();
         if (fbin > 0 && scale > 0.0f) {
           // a little below the lower edge of the bin, so that rounding cannot exclude one of its members
           const float t = __fmul_rd(__fdiv_rd((float)fbin, scale), 0.99999f);
@@ -527,29 +536,6 @@ __device__ __forceinline__ void range_sampler_role(const RowArgs& a, const Range
     SJD_PHASE(4);
     // sample(k+1) follows sample(k) after the S stages of row k-1 and itself (k >= 1)
     pos.skip(1 + cfg.stages);
-  }
-}
-
-// the instance of the sampler for this call's arguments
-template <int DTYPE, int NA, int BAR_A, bool FIRST>
-__device__ __forceinline__ void sample_rows(const RowArgs& a, const RangeCfg& cfg, const RangeSmem& sm, int tid, bool has_u,
-                                            bool has_t) {
-  if (cfg.group_rank > 0) {
-    if (has_u) {
-      if (has_t) range_sampler_role<DTYPE, true, true, true, NA, BAR_A, FIRST>(a, cfg, sm, tid);
-      else range_sampler_role<DTYPE, true, false, true, NA, BAR_A, FIRST>(a, cfg, sm, tid);
-    } else {
-      if (has_t) range_sampler_role<DTYPE, false, true, true, NA, BAR_A, FIRST>(a, cfg, sm, tid);
-      else range_sampler_role<DTYPE, false, false, true, NA, BAR_A, FIRST>(a, cfg, sm, tid);
-    }
-  } else {
-    if (has_u) {
-      if (has_t) range_sampler_role<DTYPE, true, true, false, NA, BAR_A, FIRST>(a, cfg, sm, tid);
-      else range_sampler_role<DTYPE, true, false, false, NA, BAR_A, FIRST>(a, cfg, sm, tid);
-    } else {
-      if (has_t) range_sampler_role<DTYPE, false, true, false, NA, BAR_A, FIRST>(a, cfg, sm, tid);
-      else range_sampler_role<DTYPE, false, false, false, NA, BAR_A, FIRST>(a, cfg, sm, tid);
-    }
   }
 }
 
@@ -711,7 +697,7 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
 // ---------------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------------
-template <int DTYPE, int NP, int NA>
+template <int DTYPE, int NP, int NA, bool HAS_U, bool HAS_T, bool BY_GROUPS>
 __global__ void __launch_bounds__((8 + NP + NA + 1) * 32, 1)
 rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ CUtensorMap map_c,
                    const __grid_constant__ CUtensorMap map_u) {
@@ -727,7 +713,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   extern __shared__ unsigned char smem_raw[];
   RangeSmem sm = carve_range_smem(smem_raw, cfg.mask_words);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const bool has_u = a.uncond != nullptr;
+  constexpr bool has_u = HAS_U;  // the host picks the instantiation: uncond given, 1/T != 1, thresholds by group maxima
   const float neg_inf = __int_as_float(0xff800000);
 
   if (threadIdx.x == 0) {
@@ -746,6 +732,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   }
   for (int j = threadIdx.x; j < kSampleBins; j += blockDim.x) sm.hist[j] = 0;
   for (int j = threadIdx.x; j < kSelBins; j += blockDim.x) sm.sel[j] = 0;
+  for (int j = threadIdx.x; j < kSampleBins / 32 + kSelBins / 32; j += blockDim.x) sm.hist_c[j] = 0;  // both coarse levels
   // everything above touched shared memory only; global memory is read and written from here on, so a
   // launch that was allowed to overlap the previous kernel of the stream waits for that kernel's end here
   grid_dependency_wait();
@@ -845,30 +832,24 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     return;
   }
 
-  const bool has_t = a.inv_T != 1.0f;
   if (warp < NF) {
     // ======================================= filter warps =======================================
-    if (has_u) {
-      if (has_t) range_filter_role<DTYPE, true, true>(a, cfg, sm, threadIdx.x);
-      else range_filter_role<DTYPE, true, false>(a, cfg, sm, threadIdx.x);
-    } else {
-      if (has_t) range_filter_role<DTYPE, false, true>(a, cfg, sm, threadIdx.x);
-      else range_filter_role<DTYPE, false, false>(a, cfg, sm, threadIdx.x);
-    }
+    range_filter_role<DTYPE, HAS_U, HAS_T>(a, cfg, sm, threadIdx.x);
     return;
   }
   if (warp >= NF + NP) {
     // ======================================= sampler warps =======================================
-    sample_rows<DTYPE, NA, 3, false>(a, cfg, sm, threadIdx.x - (NF + NP) * 32, has_u, has_t);
+    range_sampler_role<DTYPE, HAS_U, HAS_T, BY_GROUPS, NA, 3, false>(a, cfg, sm, threadIdx.x - (NF + NP) * 32);
     return;
   }
 
   // ======================================= finisher warps =======================================
   const int tid = threadIdx.x - NT_F;  // 0 .. NT_P-1
   // the first row's threshold, while there is nothing to finish yet
-  sample_rows<DTYPE, NP, BAR_P, true>(a, cfg, sm, tid, has_u, has_t);
+  range_sampler_role<DTYPE, HAS_U, HAS_T, BY_GROUPS, NP, BAR_P, true>(a, cfg, sm, tid);
   int flip = 0;
   bool dead = false;
+  uint32_t* const trash = reinterpret_cast<uint32_t*>(sm.ctl + kRcTrashB);
   for (int k = 0; k < n_live; ++k) {
     // from the CTA's last row on, the verification grid may be scheduled (it waits for this grid's end)
     if (k + 1 == n_live) allow_dependent_launch();
@@ -945,8 +926,12 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       code[j] = c0 | (c1 << 16);
       vmax = fmaxf(vmax, v0 ? v[j].x : neg_inf);
       vmax = fmaxf(vmax, v1 ? v[j].y : neg_inf);
-      if (c0 != 0u) atomicAdd(&sm.sel[c0 - 1u], 1u);
-      if (c1 != 0u) atomicAdd(&sm.sel[c1 - 1u], 1u);
+      // all lanes take part (a partly switched-off atomic is several times slower): code 0 counts in a word
+      // that nobody reads
+      atomicAdd(c0 != 0u ? &sm.sel[c0 - 1u] : trash, 1u);
+      atomicAdd(c0 != 0u ? &sm.sel_c[(c0 - 1u) >> 5] : trash, 1u);
+      atomicAdd(c1 != 0u ? &sm.sel[c1 - 1u] : trash, 1u);
+      atomicAdd(c1 != 0u ? &sm.sel_c[(c1 - 1u) >> 5] : trash, 1u);
     }
     // the row's maximum: per warp here, combined after the barrier
 #pragma unroll
@@ -955,20 +940,12 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     if (lane == 0) warp_max[warp - NF] = vmax;
     group_sync<NT_P, BAR_P>();
     SJD_PHASE(17);
-    // ---- exact K-th largest: threshold bin, then ranking inside it by (y descending, id ascending).  One
-    // warp searches the histogram; the others pick the result up behind a barrier.
-    if (warp == NF) {
-      const RankBin rb = warp_rank_bin<kSelBins, false>(sm.sel, (uint32_t)kcap, lane);
-      if (lane == 0) {
-        sm.ctl[kRcPBin] = rb.bin();
-        sm.ctl[kRcPAbove] = (int)rb.above;
-        sm.ctl[kRcPCount] = (int)rb.count();
-      }
-    }
-    group_sync<NT_P, BAR_P>();
-    const int tbin = sm.ctl[kRcPBin];
-    const int need = kcap - sm.ctl[kRcPAbove];  // members of the threshold bin that survive
-    const int nbin = sm.ctl[kRcPCount];
+    // ---- exact K-th largest: threshold bin, then ranking inside it by (y descending, id ascending).  Every
+    // warp searches the histogram for itself (the search is short, a barrier would cost more).
+    const RankBin rb = warp_rank_bin<kSelBins, false>(sm.sel, sm.sel_c, (uint32_t)kcap, lane);
+    const int tbin = rb.bin();
+    const int need = kcap - (int)rb.above;  // members of the threshold bin that survive
+    const int nbin = (int)rb.count();
 #pragma unroll
     for (int w = 0; w < NP; ++w) vmax = fmaxf(vmax, warp_max[w]);
     // fewer than kcap candidates (the sampled threshold was too high), a threshold bin too crowded for the
@@ -1005,18 +982,19 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       }
     }
     group_sync<NT_P, BAR_P>();
-    // one thread per member ranks it against the list: the `need` best survive (ties to the lower id), the
-    // others are marked (slot made negative)
+    // one warp per member ranks it against the list, a lane per rival: the `need` best survive (ties to the
+    // lower id), the others are marked (slot made negative)
     if (!fallback) {
-      for (int x = tid; x < nbin; x += NT_P) {
-        const BinMember me = sm.binlist[x];
-        int rank = 0;
-        for (int z = 0; z < nbin; ++z) {
+      for (int x = warp - NF; x < nbin; x += NP) {
+        const BinMember me = sm.binlist[x];  // only this warp marks member x, and only below
+        int ahead = 0;
+        for (int z = lane; z < nbin; z += 32) {
           const BinMember o = sm.binlist[z];
-          const int o_slot = o.slot < 0 ? -1 - o.slot : o.slot;  // another thread may have marked it already
-          rank += (o.y > me.y || (o.y == me.y && o_slot < me.slot)) ? 1 : 0;
+          const int o_slot = o.slot < 0 ? -1 - o.slot : o.slot;  // another warp may have marked it already
+          ahead += (o.y > me.y || (o.y == me.y && o_slot < me.slot)) ? 1 : 0;
         }
-        if (rank >= need) sm.binlist[x].slot = -1 - me.slot;
+        const int rank = __reduce_add_sync(0xffffffffu, ahead);
+        if (lane == 0 && rank >= need) sm.binlist[x].slot = -1 - me.slot;
       }
     }
     group_sync<NT_P, BAR_P>();
@@ -1074,6 +1052,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     if (fallback) {
       // redone by the any-shape path after the last row; the bins must be clear again for the next one
       for (int j = tid; j < kSelBins; j += NT_P) sm.sel[j] = 0;
+      if (tid < kSelBins / 32) sm.sel_c[tid] = 0;
       if (tid == 0) sm.redo[sm.ctl[kRcRedo]++] = row;
       group_sync<NT_P, BAR_P>();
       continue;
@@ -1093,6 +1072,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     // these words of st_ids are this thread's share of sel: zero again for the next row
 #pragma unroll
     for (int x = 0; x < kFinItems / 4; ++x) *reinterpret_cast<uint4*>(sm.sel + k0 + 4 * x) = make_uint4(0u, 0u, 0u, 0u);
+    if (tid < kSelBins / 32) sm.sel_c[tid] = 0;
     const float Z = group_sum1_f32<NT_P, BAR_P>(zpart, tid, sm.scan_p, flip);
     SJD_PHASE(21);
     int32_t* out_ids = a.out_ids + (size_t)row * kcap;

@@ -227,15 +227,34 @@ cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
 constexpr int kSamplerWarps = 3;
 constexpr int kRangeFinisherWarps = 16;
 
-template <int DTYPE>
-cudaError_t launch_ranges(const sjd::RowArgs& ra, const sjd::RangeCfg& cfg, const CUtensorMap& mc, const CUtensorMap& mu,
-                          size_t smem, int grid, cudaStream_t st) {
-  auto kern = sjd::rows_ranges_kernel<DTYPE, kRangeFinisherWarps, kSamplerWarps>;
+// One kernel per logits type and per combination of (guidance given, temperature applied, thresholds by
+// group maxima): each holds only the code its launch runs, which matters because the roles' code does not fit
+// the instruction caches comfortably.
+template <int DTYPE, bool HAS_U, bool HAS_T, bool BY_GROUPS>
+cudaError_t launch_ranges_as(const sjd::RowArgs& ra, const sjd::RangeCfg& cfg, const CUtensorMap& mc, const CUtensorMap& mu,
+                             size_t smem, int grid, cudaStream_t st) {
+  auto kern = sjd::rows_ranges_kernel<DTYPE, kRangeFinisherWarps, kSamplerWarps, HAS_U, HAS_T, BY_GROUPS>;
   static sjd::DeviceOnce configured;  // per instantiation
   const cudaError_t e = allow_large_smem(kern, configured, (int)kSmemLimit);
   if (e != cudaSuccess) return e;
   return launch_after(kern, dim3((unsigned)grid), dim3((8 + kRangeFinisherWarps + kSamplerWarps + 1) * 32), smem, st, true, ra,
                       cfg, mc, mu);
+}
+
+template <int DTYPE>
+cudaError_t launch_ranges(const sjd::RowArgs& ra, const sjd::RangeCfg& cfg, const CUtensorMap& mc, const CUtensorMap& mu,
+                          size_t smem, int grid, cudaStream_t st) {
+  const int which = (ra.uncond != nullptr ? 4 : 0) | (ra.inv_T != 1.0f ? 2 : 0) | (cfg.group_rank > 0 ? 1 : 0);
+  switch (which) {
+    case 0: return launch_ranges_as<DTYPE, false, false, false>(ra, cfg, mc, mu, smem, grid, st);
+    case 1: return launch_ranges_as<DTYPE, false, false, true>(ra, cfg, mc, mu, smem, grid, st);
+    case 2: return launch_ranges_as<DTYPE, false, true, false>(ra, cfg, mc, mu, smem, grid, st);
+    case 3: return launch_ranges_as<DTYPE, false, true, true>(ra, cfg, mc, mu, smem, grid, st);
+    case 4: return launch_ranges_as<DTYPE, true, false, false>(ra, cfg, mc, mu, smem, grid, st);
+    case 5: return launch_ranges_as<DTYPE, true, false, true>(ra, cfg, mc, mu, smem, grid, st);
+    case 6: return launch_ranges_as<DTYPE, true, true, false>(ra, cfg, mc, mu, smem, grid, st);
+    default: return launch_ranges_as<DTYPE, true, true, true>(ra, cfg, mc, mu, smem, grid, st);
+  }
 }
 
 template <int DTYPE>
