@@ -77,8 +77,7 @@ constexpr size_t kSmemLimit = 227u * 1024u;
 // is at most Poisson(a)-distributed (drawing without replacement only narrows it), so m = a + z sqrt(m),
 // i.e. sqrt(m) = z/2 + sqrt(z^2/4 + a), leaves the threshold above the true one (too few candidates, the
 // row redone by the any-shape path at many times the cost) with a probability below 4e-6 per row at z = 4.5.
-int sample_rank(double a) {
-  constexpr double z = 4.5;
+int sample_rank(double a, double z = 4.5) {
   const double root = z / 2 + std::sqrt(z * z / 4 + a);
   return (int)std::ceil(root * root);
 }
@@ -160,9 +159,21 @@ bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem
   if (mask_words > sjd::kMaskWordsMax) return false;
   const int n_sample = sjd::kRangeThreads * bw;
   const double a = (double)kcap / S;
-  const int m = sample_rank(a);
+  int m = sample_rank(a);
   if (m > n_sample / 2) return false;
-  const int sample_all = m > n_sample / 8 ? 1 : 0;  // the rank must exist among what the first pass bins
+  // The element rank m can be taken as a rank among the maxima of the sample's groups of eight (see the
+  // sampler): directly while at most a tenth of the sample lies above the threshold.  Up to a fifth the group
+  // maxima still resolve the rank, but up to 1.6 times less sharply than the elements would: a margin of 6.5
+  // instead of 4.5 standard deviations keeps the row at least as safe.  Beyond that every element is binned.
+  bool by_groups = m <= n_sample / 8 && (double)m / n_sample <= 0.10;
+  if (!by_groups) {
+    const int m_wide = sample_rank(a, 6.5);
+    if ((double)m_wide / n_sample <= 0.20) {
+      m = m_wide;
+      by_groups = true;
+    }
+  }
+  const int sample_all = m > n_sample / 8 ? 1 : 0;  // the rank must exist among what an element-wise first pass bins
   // candidates of a row: m S on average; pairs of neighbours with at least one candidate: a little fewer
   const double cand = (double)m * S, cand_sd = (double)S * std::sqrt((double)m);
   const double thin = 1.0 - 0.5 * cand / V;
@@ -173,11 +184,9 @@ bool plan_ranges(const sjd_params* P, int kcap, sjd::RangeCfg* cfg, size_t* smem
   if (need_encoder && encode_tiled_fn() == nullptr) return false;
   cfg->sample_rank = m;
   cfg->sample_all = sample_all;
-  // the element rank m as a rank among the maxima of the sample's groups of eight (see the sampler); only
-  // while at most a tenth of the sample lies above the threshold, beyond that the group maxima resolve it badly
   {
     const double p = (double)m / n_sample, groups = n_sample / 8.0;
-    cfg->group_rank = (!sample_all && p <= 0.10) ? (int)std::ceil(groups * (1.0 - std::pow(1.0 - p, 8.0))) : 0;
+    cfg->group_rank = by_groups ? (int)std::ceil(groups * (1.0 - std::pow(1.0 - p, 8.0))) : 0;
   }
   cfg->stages = S;
   cfg->range_len = R;
