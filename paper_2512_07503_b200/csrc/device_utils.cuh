@@ -156,6 +156,11 @@ __device__ __forceinline__ bool group_any(bool pred) {
   return r != 0;
 }
 
+__device__ __forceinline__ uint64_t shfl_u64(uint64_t v, int src) {
+  const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)v, src);
+  const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)(v >> 32), src);
+  return (uint64_t)lo | ((uint64_t)hi << 32);
+}
 __device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int d) {
   const uint32_t lo = __shfl_up_sync(0xffffffffu, (uint32_t)v, d);
   const uint32_t hi = __shfl_up_sync(0xffffffffu, (uint32_t)(v >> 32), d);
@@ -314,12 +319,24 @@ __device__ __forceinline__ T group_scan1(T v, int tid, uint64_t* scratch, int& f
   flip ^= 1;
   if (lane == 31) bank[warp] = (uint64_t)inc;
   group_sync<NT, BAR>();
-  T base = 0, tot = 0;
+  // every warp scans the warps' totals for itself, lane w holding warp w's (a walk over the NW words by
+  // every thread costs several times the instructions)
+  const T x = lane < NW ? (T)bank[lane] : (T)0;
+  T xi = x;
 #pragma unroll
-  for (int w = 0; w < NW; ++w) {
-    const T x = (T)bank[w];
-    tot += x;
-    if (w < warp) base += x;
+  for (int d = 1; d < NW; d <<= 1) {
+    T n;
+    if (sizeof(T) == 8) n = (T)shfl_up_u64((uint64_t)xi, d);
+    else n = (T)__shfl_up_sync(0xffffffffu, (uint32_t)xi, d);
+    if (lane >= d) xi += n;
+  }
+  T tot, base;
+  if (sizeof(T) == 8) {
+    tot = (T)shfl_u64((uint64_t)xi, NW - 1);
+    base = (T)shfl_u64((uint64_t)(xi - x), warp);
+  } else {
+    tot = (T)__shfl_sync(0xffffffffu, (uint32_t)xi, NW - 1);
+    base = (T)__shfl_sync(0xffffffffu, (uint32_t)(xi - x), warp);
   }
   *total = tot;
   return base + inc - v;
@@ -337,6 +354,13 @@ __device__ __forceinline__ float group_sum1_f32(float v, int tid, uint64_t* scra
   flip ^= 1;
   if (lane == 0) bank[warp] = v;
   group_sync<NT, BAR>();
+  if ((NW & (NW - 1)) == 0) {
+    // lane l takes warp (l mod NW)'s sum; the butterfly adds the same pairs in every lane and every warp
+    float t = bank[lane & (NW - 1)];
+#pragma unroll
+    for (int d = NW / 2; d > 0; d >>= 1) t += __shfl_xor_sync(0xffffffffu, t, d);
+    return t;
+  }
   float t = 0.0f;
 #pragma unroll
   for (int w = 0; w < NW; ++w) t += bank[w];
