@@ -709,7 +709,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   constexpr int NS = kRangeRingStages;
   constexpr int BW = 64 / (DTYPE != 0 ? 2 : 4);  // elements per stage and range
   static_assert(NT_F == NF * 32 && kFinItems * NT_P == kKcapMax && (kFinItems == 4 || kFinItems == 8), "group sizes");
-  static_assert(2 * kPairChunk <= 32 && NP <= 16, "hit bits in one word; warp maxima in the spare scratch slots");
+  static_assert(2 * kPairChunk <= 32 && NP <= 16 && (NP & (NP - 1)) == 0, "hit bits in one word; warp maxima in the spare scratch slots");
   extern __shared__ unsigned char smem_raw[];
   RangeSmem sm = carve_range_smem(smem_raw, cfg.mask_words);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -946,27 +946,31 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     const int tbin = rb.bin();
     const int need = kcap - (int)rb.above;  // members of the threshold bin that survive
     const int nbin = (int)rb.count();
+    // lane l takes warp (l mod NP)'s maximum; the butterfly leaves the row's maximum in every lane
+    vmax = warp_max[lane & (NP - 1)];
 #pragma unroll
-    for (int w = 0; w < NP; ++w) vmax = fmaxf(vmax, warp_max[w]);
+    for (int d = NP / 2; d > 0; d >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, d));
     // fewer than kcap candidates (the sampled threshold was too high), a threshold bin too crowded for the
     // on-chip ranking, or no finite maximum: the any-shape path redoes the row
     if (tbin < 0 || nbin > kBinListCap || !(vmax <= 3.402823466e38f)) fallback = true;
     SJD_PHASE(18);
     const uint32_t tcode = (uint32_t)tbin + 1u;
-    uint32_t n_above = 0;
-    uint32_t hits = 0;  // bit 2j + h: value h of pair j lies in the threshold bin
+    uint32_t above = 0;  // bit 2j + h: value h of pair j lies in a bin above the threshold bin
+    uint32_t hits = 0;   // likewise: it lies in the threshold bin
     int my_at0 = -1, my_at1 = -1;
     bool many = false;
     if (!fallback) {
 #pragma unroll
       for (int j = 0; j < kPairChunk; ++j) {
         const uint32_t c0 = code[j] & 0xffffu, c1 = code[j] >> 16;
-        n_above += (c0 > tcode ? 1u : 0u) + (c1 > tcode ? 1u : 0u);
+        above |= (c0 > tcode ? 1u : 0u) << (2 * j);
+        above |= (c1 > tcode ? 1u : 0u) << (2 * j + 1);
         hits |= (c0 == tcode ? 1u : 0u) << (2 * j);
         hits |= (c1 == tcode ? 1u : 0u) << (2 * j + 1);
       }
       // the members of the threshold bin (a handful per row) go on a list: value and position in the pair
       // list; the thread remembers where its first two went
+      if (hits != 0u) {
 #pragma unroll
       for (int j = 0; j < kPairChunk; ++j) {
 #pragma unroll
@@ -979,6 +983,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
             else many = true;
           }
         }
+      }
       }
     }
     group_sync<NT_P, BAR_P>();
@@ -1020,18 +1025,12 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     }
     SJD_PHASE(19);
     uint32_t total_alive;
-    uint32_t out_pos = group_scan1<NT_P, BAR_P, uint32_t>(n_above + (uint32_t)__popc(hits), tid, sm.scan_p, flip, &total_alive);
+    uint32_t out_pos = group_scan1<NT_P, BAR_P, uint32_t>((uint32_t)__popc(above | hits), tid, sm.scan_p, flip, &total_alive);
     if (!fallback && total_alive != (uint32_t)kcap) fallback = true;  // cannot happen; keep the result exact anyway
     if (!fallback) {
       // ---- survivors, already in ascending id order (this overwrites sel and the member list).  The
       // position of each follows from the bits of those before it, so the stores do not wait for one another.
-      uint32_t alive = hits;
-#pragma unroll
-      for (int j = 0; j < kPairChunk; ++j) {
-        const uint32_t c0 = code[j] & 0xffffu, c1 = code[j] >> 16;
-        alive |= (c0 > tcode ? 1u : 0u) << (2 * j);
-        alive |= (c1 > tcode ? 1u : 0u) << (2 * j + 1);
-      }
+      const uint32_t alive = hits | above;
 #pragma unroll
       for (int j = 0; j < kPairChunk; ++j) {
         const int id = 2 * (int)((qq[j >> 1] >> (16 * (j & 1))) & 0xffffu);
