@@ -884,19 +884,26 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     // ---- every thread takes an equal share of the pair list into registers: a run of consecutive pairs, so
     // that concatenating the threads' survivors keeps the id order.  The list then goes straight back to the
     // filter warps, which may already be waiting to write the next row's.
-    const uint32_t chunk = fallback ? 0u : (n_pairs + NT_P - 1) / NT_P;  // <= kPairChunk
-    const uint32_t my_first = min((uint32_t)tid * chunk, n_pairs);
-    const uint32_t my_count = fallback ? 0u : min(my_first + chunk, n_pairs) - my_first;
+    // The shares differ by one pair at most (the first n mod NT threads take one more), and a warp skips the
+    // slots none of its threads fills: with 2,600 pairs most warps work on five slots, not on all seven.
+    const uint32_t share = fallback ? 0u : n_pairs / NT_P, extra = fallback ? 0u : n_pairs % NT_P;
+    const uint32_t my_first = (uint32_t)tid * share + min((uint32_t)tid, extra);
+    const uint32_t my_count = share + ((uint32_t)tid < extra ? 1u : 0u);          // <= kPairChunk
+    const uint32_t wcount = share + (((uint32_t)tid & ~31u) < extra ? 1u : 0u);  // the warp's largest share
     float2 v[kPairChunk];
     uint32_t qq[(kPairChunk + 1) / 2];  // pair numbers, two to a word
 #pragma unroll
+    for (int j = 0; j < (kPairChunk + 1) / 2; ++j) qq[j] = 0u;
+#pragma unroll
     for (int j = 0; j < kPairChunk; ++j) {
-      // a slot beyond the thread's share reads a valid address and is masked out below
-      const uint32_t at = min(my_first + (uint32_t)j, (uint32_t)kRangePairCap - 1u);
-      v[j] = *reinterpret_cast<const float2*>(&sm.pair_y[at]);
-      const uint32_t q = sm.pair_q[at];
-      if ((j & 1) == 0) qq[j >> 1] = q;
-      else qq[j >> 1] |= q << 16;
+      if ((uint32_t)j < wcount) {
+        // a slot beyond the thread's share reads a valid address and is masked out below
+        const uint32_t at = min(my_first + (uint32_t)j, (uint32_t)kRangePairCap - 1u);
+        v[j] = *reinterpret_cast<const float2*>(&sm.pair_y[at]);
+        const uint32_t q = sm.pair_q[at];
+        if ((j & 1) == 0) qq[j >> 1] = q;
+        else qq[j >> 1] |= q << 16;
+      }
     }
     if (tid == 0) {
       sm.ctl[kRcGather] = 0;
@@ -918,6 +925,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     float vmax = neg_inf;
 #pragma unroll
     for (int j = 0; j < kPairChunk; ++j) {
+      if ((uint32_t)j >= wcount) continue;
       const bool mine = (uint32_t)j < my_count;
       const bool v0 = mine && v[j].x >= tau0, v1 = mine && v[j].y >= tau0;  // false for NaN
       const int q0 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[j].x, tau0), scale)), kSelBins - 1);
@@ -962,6 +970,7 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     if (!fallback) {
 #pragma unroll
       for (int j = 0; j < kPairChunk; ++j) {
+        if ((uint32_t)j >= wcount) continue;
         const uint32_t c0 = code[j] & 0xffffu, c1 = code[j] >> 16;
         above |= (c0 > tcode ? 1u : 0u) << (2 * j);
         above |= (c1 > tcode ? 1u : 0u) << (2 * j + 1);
@@ -1028,22 +1037,27 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     uint32_t out_pos = group_scan1<NT_P, BAR_P, uint32_t>((uint32_t)__popc(above | hits), tid, sm.scan_p, flip, &total_alive);
     if (!fallback && total_alive != (uint32_t)kcap) fallback = true;  // cannot happen; keep the result exact anyway
     if (!fallback) {
-      // ---- survivors, already in ascending id order (this overwrites sel and the member list).  The
-      // position of each follows from the bits of those before it, so the stores do not wait for one another.
+      // ---- survivors, already in ascending id order (this overwrites sel and the member list)
       const uint32_t alive = hits | above;
+      // one cursor walks through both staging arrays (the values sit kKcapMax words behind the ids): a
+      // survivor is stored and moves the cursor on, everything else is predicated off
+      static_assert(kKcapMax * 4 == 8192, "offset of st_vals behind st_ids in the store below");
+      uint32_t at = smem_u32(sm.st_ids) + out_pos * 4u;
+      auto stage_if = [&at](uint32_t id, float val, uint32_t bit) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %3, 0;\n\t@p st.shared.u32 [%0], %1;\n\t@p st.shared.f32 [%0+8192], %2;\n\t"
+            "@p add.u32 %0, %0, 4;\n\t}"
+            : "+r"(at)
+            : "r"(id), "f"(val), "r"(bit)
+            : "memory");
+      };
 #pragma unroll
       for (int j = 0; j < kPairChunk; ++j) {
-        const int id = 2 * (int)((qq[j >> 1] >> (16 * (j & 1))) & 0xffffu);
-        const uint32_t at0 = out_pos + (uint32_t)__popc(alive & ((1u << (2 * j)) - 1u));
-        const uint32_t at1 = out_pos + (uint32_t)__popc(alive & ((1u << (2 * j + 1)) - 1u));
-        if ((alive >> (2 * j)) & 1u) {
-          sm.st_ids[at0] = id;
-          sm.st_vals[at0] = canonical(v[j].x);
-        }
-        if ((alive >> (2 * j + 1)) & 1u) {
-          sm.st_ids[at1] = id + 1;
-          sm.st_vals[at1] = canonical(v[j].y);
-        }
+        if ((uint32_t)j >= wcount) continue;
+        const uint32_t id = 2u * ((j & 1) ? qq[j >> 1] >> 16 : qq[j >> 1] & 0xffffu);
+        // a survivor is neither a NaN nor below tau0: adding zero is all that is left of canonical()
+        stage_if(id, __fadd_rn(v[j].x, 0.0f), alive & (1u << (2 * j)));
+        stage_if(id + 1u, __fadd_rn(v[j].y, 0.0f), alive & (2u << (2 * j)));
       }
     }
     group_sync<NT_P, BAR_P>();
