@@ -849,7 +849,6 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
   range_sampler_role<DTYPE, HAS_U, HAS_T, BY_GROUPS, NP, BAR_P, true>(a, cfg, sm, tid);
   int flip = 0;
   bool dead = false;
-  uint32_t* const trash = reinterpret_cast<uint32_t*>(sm.ctl + kRcTrashB);
   for (int k = 0; k < n_live; ++k) {
     // from the CTA's last row on, the verification grid may be scheduled (it waits for this grid's end)
     if (k + 1 == n_live) allow_dependent_launch();
@@ -916,11 +915,13 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       if (tid == 0) sm.redo[sm.ctl[kRcRedo]++] = row;  // redone by the any-shape path after the last row
       continue;
     }
-    // ---- linear bins over [tau0, top] (top: the largest sample value; anything above it lands in the last
-    // bin); monotone in y, so a higher bin never holds a smaller value.  A thread keeps the bins of its values
-    // in registers: 0 = below tau0 (not a candidate), otherwise bin + 1.
+    // ---- linear bins 1 .. kSelBins - 1 over [tau0, top] (top: the largest sample value; anything above it
+    // lands in the last bin); monotone in y, so a higher bin never holds a smaller value.  Bin 0 takes what is
+    // no candidate (below tau0, NaN, a slot beyond the thread's share): every lane of every update is on (a
+    // partly switched-off atomic is several times slower, lanes that meet in one word cost nothing) and no
+    // address has to be chosen.  A thread keeps the bins of its values in registers.
     const float range = __fsub_rn(top, tau0);
-    const float scale = range > 0.0f ? __fdiv_rn((float)kSelBins * 0.999f, range) : 0.0f;
+    const float scale = range > 0.0f ? __fdiv_rn((float)(kSelBins - 1) * 0.999f, range) : 0.0f;
     uint32_t code[kPairChunk];
     float vmax = neg_inf;
 #pragma unroll
@@ -928,18 +929,16 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       if ((uint32_t)j >= wcount) continue;
       const bool mine = (uint32_t)j < my_count;
       const bool v0 = mine && v[j].x >= tau0, v1 = mine && v[j].y >= tau0;  // false for NaN
-      const int q0 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[j].x, tau0), scale)), kSelBins - 1);
-      const int q1 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[j].y, tau0), scale)), kSelBins - 1);
+      const int q0 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[j].x, tau0), scale)), kSelBins - 2);
+      const int q1 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[j].y, tau0), scale)), kSelBins - 2);
       const uint32_t c0 = v0 ? (uint32_t)q0 + 1u : 0u, c1 = v1 ? (uint32_t)q1 + 1u : 0u;
       code[j] = c0 | (c1 << 16);
       vmax = fmaxf(vmax, v0 ? v[j].x : neg_inf);
       vmax = fmaxf(vmax, v1 ? v[j].y : neg_inf);
-      // all lanes take part (a partly switched-off atomic is several times slower): code 0 counts in a word
-      // that nobody reads
-      atomicAdd(c0 != 0u ? &sm.sel[c0 - 1u] : trash, 1u);
-      atomicAdd(c0 != 0u ? &sm.sel_c[(c0 - 1u) >> 5] : trash, 1u);
-      atomicAdd(c1 != 0u ? &sm.sel[c1 - 1u] : trash, 1u);
-      atomicAdd(c1 != 0u ? &sm.sel_c[(c1 - 1u) >> 5] : trash, 1u);
+      atomicAdd(&sm.sel[c0], 1u);
+      atomicAdd(&sm.sel_c[c0 >> 5], 1u);
+      atomicAdd(&sm.sel[c1], 1u);
+      atomicAdd(&sm.sel_c[c1 >> 5], 1u);
     }
     // the row's maximum: per warp here, combined after the barrier
 #pragma unroll
@@ -960,9 +959,9 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
     for (int d = NP / 2; d > 0; d >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, d));
     // fewer than kcap candidates (the sampled threshold was too high), a threshold bin too crowded for the
     // on-chip ranking, or no finite maximum: the any-shape path redoes the row
-    if (tbin < 0 || nbin > kBinListCap || !(vmax <= 3.402823466e38f)) fallback = true;
+    if (tbin <= 0 || nbin > kBinListCap || !(vmax <= 3.402823466e38f)) fallback = true;  // bin 0: the rank lies among what is no candidate
     SJD_PHASE(18);
-    const uint32_t tcode = (uint32_t)tbin + 1u;
+    const uint32_t tcode = (uint32_t)tbin;  // a value's code is its bin
     uint32_t above = 0;  // bit 2j + h: value h of pair j lies in a bin above the threshold bin
     uint32_t hits = 0;   // likewise: it lies in the threshold bin
     int my_at0 = -1, my_at1 = -1;
