@@ -655,10 +655,8 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
     const bool fallback = ((sum >> 14) & 0x1ffu) != 0u || n_pairs > (uint32_t)kRangePairCap;
     SJD_PHASE(11);
     if (!fallback) {
-      uint32_t qn = (uint32_t)(tid * (cfg.range_len >> 1));  // pair number of the first bit of the current mask word
-      uint32_t y_at = smem_u32(sm.pair_y) + my_off * 8u, q_at = smem_u32(sm.pair_q) + my_off * 2u;
-      int w = 0;
-      uint32_t x = ~sm.masks[tid];
+      // (1) the pairs, four at a time: loads and stores of different entries do not wait for one another
+      uint32_t y_at = smem_u32(sm.pair_y) + my_off * 8u;
       for (int e0 = 0; e0 < n_e; e0 += 4) {
         uint64_t v[4];
 #pragma unroll
@@ -666,20 +664,25 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
           asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v[u]) : "r"(list_base + (uint32_t)min(e0 + u, kRangeListCap - 1) * kStride));
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          if (e0 + u < n_e) {
-            while (x == 0u && w + 1 < mask_words) {
-              ++w;
-              qn += 32u;
-              x = ~sm.masks[(size_t)w * NT_F + tid];
-            }
-            const uint32_t bitpos = (uint32_t)__clz((int)x);
-            x &= ~(0x80000000u >> bitpos);
-            asm volatile("st.shared.b64 [%0], %1;" ::"r"(y_at), "l"(v[u]) : "memory");
-            asm volatile("st.shared.u16 [%0], %1;" ::"r"(q_at), "h"((uint16_t)(qn + bitpos)) : "memory");
-            y_at += 8u;
-            q_at += 2u;
-          }
+          if (e0 + u < n_e) asm volatile("st.shared.b64 [%0], %1;" ::"r"(y_at + 8u * (uint32_t)u), "l"(v[u]) : "memory");
         }
+        y_at += 32u;
+      }
+      // (2) their pair numbers: the set hit bits, word by word.  The walk over the words is the same for
+      // every thread of the warp (one mask load per word, outside the inner loop); only the number of bits
+      // in a word differs from lane to lane.  (With the word change inside a per-entry loop every entry paid
+      // for a divergent branch and a shared-memory load: the drain took three times as long.)
+      uint32_t q_at = smem_u32(sm.pair_q) + my_off * 2u;
+      uint32_t qn = (uint32_t)(tid * (cfg.range_len >> 1));  // pair number of the first bit of the current mask word
+      for (int w = 0; w < mask_words; ++w) {
+        uint32_t x = ~sm.masks[(size_t)w * NT_F + tid];
+        while (x != 0u) {
+          const uint32_t bitpos = (uint32_t)__clz((int)x);
+          x &= ~(0x80000000u >> bitpos);
+          asm volatile("st.shared.u16 [%0], %1;" ::"r"(q_at), "h"((uint16_t)(qn + bitpos)) : "memory");
+          q_at += 2u;
+        }
+        qn += 32u;
       }
     }
     if (tid == 0) {
