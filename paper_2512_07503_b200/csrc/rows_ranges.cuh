@@ -3,13 +3,17 @@
 // One persistent CTA per SM, rows round-robin, four roles:
 //
 //   producer (1 warp)   streams rows through a ring of shared-memory stages with tiled TMA copies.
-//   sampler (4 warps)   works one row AHEAD of the filter: it gets a copy of the next row's stage 0 (a
+//   sampler (3 warps)   works one row AHEAD of the filter: it gets a copy of the next row's stage 0 (a
 //                       systematic sample of that row) through the ring, and turns it into the candidate
 //                       threshold tau0 of that row while the filter warps are still streaming the current one.
 //   filter (8 warps)    merges the staged pairs into logits y and keeps the pairs that reach tau0; at the end
 //                       of the row it compacts its lists into a dense candidate list in ascending id order.
-//   finisher (8 warps)  one row BEHIND the filter: exact K-th largest among the candidates, softmax, output,
-//                       the row's own draw.
+//   finisher (16 warps) one row BEHIND the filter: exact K-th largest among the candidates, softmax, output,
+//                       the row's own draw.  Before the CTA's first row they compute that row's threshold.
+//
+// Every combination of (guidance given, temperature applied, thresholds by group maxima or by elements) is a
+// kernel of its own, chosen on the host: the roles' code is large against the SM's instruction caches, and
+// the variants a launch does not run cost time merely by lying between those it does.
 //
 // The row of V logits is viewed as a matrix of 256 ranges x R ids (R = V/256): filter thread t owns ids
 // [t R, (t+1) R).  A ring stage is a column slice of that matrix, 64 bytes per range, fetched by ONE tiled
