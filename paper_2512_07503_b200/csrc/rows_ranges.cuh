@@ -257,6 +257,15 @@ __device__ __forceinline__ void tma_load_box(void* dst, const CUtensorMap* map, 
       : "memory");
 }
 
+// The same box asked into the L2 only, ahead of its copy: the ring's three stages cannot cover the latency of
+// HBM under load (a stage comes back 3-4 K cycles after its slot was given up and is worked through in 1.3 K),
+// the L2's they can.
+__device__ __forceinline__ void tma_prefetch_box(const CUtensorMap* map, int x, int z) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(reinterpret_cast<uint64_t>(map)),
+               "r"(x), "r"(0), "r"(z)
+               : "memory");
+}
+
 // Histograms come in two levels: BINS fine bins and BINS / 32 coarse ones, coarse[c] counting what fine bins
 // 32 c .. 32 c + 31 count (whoever adds to a fine bin adds to its coarse bin as well: shared-memory atomics
 // that ask for no old value are cheap, a long search by one warp while the others wait is not).
@@ -578,8 +587,8 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
     uint32_t cur = list_base;  // shared-memory address of the thread's next free entry
     uint32_t imw = 0;          // inverted hit bits of the groups filtered since the last full mask word
     bool overflow = false;
-    // One group: four pairs.  A pair is always stored at the cursor; the cursor moves on only for a hit,
-    // i.e. when max(pair) >= thr.  A pair of NaNs and -inf never hit.
+    // One group: four pairs.  A pair is stored at the cursor, and the cursor moves on, only for a hit, i.e.
+    // when max(pair) >= thr.  A pair of NaNs and -inf never hit.
     auto filter_group = [&](const RawTile<DTYPE>& raw, float thr) {
       float y[8];
       merge_raw<DTYPE, HAS_U, HAS_T>(raw, s2, t2, y);
@@ -592,11 +601,15 @@ __device__ __forceinline__ void range_filter_role(const RowArgs& a, const RangeC
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const float m = fmaxf(y[2 * q], y[2 * q + 1]);
-        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(d), "f"(y[2 * q]), "f"(y[2 * q + 1]) : "memory");
-        // hit: the cursor moves on; miss: the pair's bit is set in the inverted mask (both predicated, no branch)
-        asm("{\n\t.reg .pred p;\n\tsetp.ge.f32 p, %2, %3;\n\t@p add.u32 %0, %0, %4;\n\t@!p or.b32 %1, %1, %5;\n\t}"
+        // hit: the pair is stored and the cursor moves on; miss: the pair's bit is set in the inverted mask
+        // (all predicated, no branch).  A store with no lane on costs shared memory nothing, one with two or
+        // three lanes on one pass instead of the two a full warp's 256 bytes take.
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ge.f32 p, %2, %3;\n\t@p st.shared.v2.f32 [%0], {%6, %7};\n\t@p add.u32 %0, %0, %4;\n\t"
+            "@!p or.b32 %1, %1, %5;\n\t}"
             : "+r"(d), "+r"(imw)
-            : "f"(m), "f"(thr), "r"(kStride), "r"(8u >> q));
+            : "f"(m), "f"(thr), "r"(kStride), "r"(8u >> q), "f"(y[2 * q]), "f"(y[2 * q + 1])
+            : "memory");
       }
       cur = d;
     };
@@ -819,11 +832,26 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       if (has_u) tma_load_box(dst + kRangeStageBytes, &map_u, x, row, bar);
       pos.step();
     };
-    if (n_live > 0) issue(0, sm.tab[0].row, 0);
+    auto prefetch = [&](int x, int row) {
+      tma_prefetch_box(&map_c, x, row);
+      if (has_u) tma_prefetch_box(&map_u, x, row);
+    };
+    if (n_live > 0) {
+      issue(0, sm.tab[0].row, 0);
+    }
     for (int k = 0; k < n_live && ok; ++k) {
       if (k + 1 < n_live) issue(0, sm.tab[k + 1].row, k + 1);
       const int row = sm.tab[k].row;
-      for (int s = 0; s < cfg.stages && ok; ++s) issue(s * BW, row, -1);
+      for (int s = 0; s < cfg.stages && ok; ++s) {
+        // the stage that will take this stage's slot next is asked into the L2 now (stage 0 of a row comes
+        // with that row's sample)
+        {
+          const int ahead = s + NS;
+          if (ahead < cfg.stages) prefetch(ahead * BW, row);
+          else if (k + 1 < n_live && ahead - cfg.stages > 0 && ahead - cfg.stages < cfg.stages) prefetch((ahead - cfg.stages) * BW, sm.tab[k + 1].row);
+        }
+        issue(s * BW, row, -1);
+      }
     }
     // drain: every copy armed here must have landed before the CTA may exit.  The latest copy into a slot
     // is the only one that can still be in flight; a slot whose latest copy was a sample holds the latest
