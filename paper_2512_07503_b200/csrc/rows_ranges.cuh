@@ -931,8 +931,9 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
 #pragma unroll
     for (int j = 0; j < kPairChunk; ++j) {
       if ((uint32_t)j < wcount) {
-        // a slot beyond the thread's share reads a valid address and is masked out below
-        const uint32_t at = min(my_first + (uint32_t)j, (uint32_t)kRangePairCap - 1u);
+        // a slot beyond the thread's share reads another pair of this row (the next thread's, or the row's
+        // last) and is masked out below - except for the row's maximum, which it cannot raise
+        const uint32_t at = min(my_first + (uint32_t)j, n_pairs - 1u);  // wcount > 0, so the row has pairs
         v[j] = *reinterpret_cast<const float2*>(&sm.pair_y[at]);
         const uint32_t q = sm.pair_q[at];
         if ((j & 1) == 0) qq[j >> 1] = q;
@@ -968,8 +969,9 @@ rows_ranges_kernel(const RowArgs a, const RangeCfg cfg, const __grid_constant__ 
       const int q1 = min(__float2int_rd(__fmul_rn(__fsub_rn(v[j].y, tau0), scale)), kSelBins - 2);
       const uint32_t c0 = v0 ? (uint32_t)q0 + 1u : 0u, c1 = v1 ? (uint32_t)q1 + 1u : 0u;
       code[j] = c0 | (c1 << 16);
-      vmax = fmaxf(vmax, v0 ? v[j].x : neg_inf);
-      vmax = fmaxf(vmax, v1 ? v[j].y : neg_inf);
+      // the largest candidate is the largest value of the list (a NaN is passed over, a value below tau0
+      // lies below every candidate, and a row without candidates is redone anyway)
+      vmax = max3(vmax, v[j].x, v[j].y);
       atomicAdd(&sm.sel[c0], 1u);
       atomicAdd(&sm.sel_c[c0 >> 5], 1u);
       atomicAdd(&sm.sel[c1], 1u);
