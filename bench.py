@@ -331,7 +331,7 @@ def run_ours(args):
 
 # DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture, per workload;
 # the capture is summarised under profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES = {"cfg4": 281_100_000}
+NCU_TRAFFIC_BYTES = {"cfg4": 281_000_000}
 NCU_TRAFFIC_SOURCE = ("stored figure, not measured by this run: dram__bytes_read.sum + dram__bytes_write.sum of one launch, "
                       "from the ncu capture summarised in profiles/rows_ranges_cfg4.md")
 
